@@ -1,0 +1,174 @@
+/*
+ * dba.h -- C ABI of the Dynamic Beam Allocation step library (CUDA, sm_100a).
+ *
+ * The library runs, for a batch of B independent sentences with beam size k and vocabulary V, the
+ * per-timestep step of lexically constrained beam search with dynamic beam allocation
+ * (Post & Vilar 2018: Algorithm 2 "KBEST-DBA", Sections 3.1-3.3) with the log-softmax of Section 2 in
+ * front of it.  All arithmetic of the step runs in CUDA kernels; there is no CPU fallback.
+ *
+ * Conventions
+ *   - Every function returns a dba_status; nothing throws or aborts.  Argument errors are detected on
+ *     the host before anything is launched.
+ *   - "dev" pointers are device memory, "host" pointers are host memory.  The library allocates no
+ *     device memory: the caller provides one workspace (dba_workspace_bytes) that must outlive the
+ *     handle, and owns every input and output buffer.  The library owns only the handle.
+ *   - dba_step only enqueues work on the stream given to dba_init and does not synchronise.
+ *   - Row r = b*k + h of any [B*k, ...] array belongs to beam slot h of sentence b.
+ *   - Token ids are int32 in [0, V).  pad_id / bos_id / eos_id are the special symbols.
+ *   - Logits must be finite or -inf.  NaN or +inf input is undefined behaviour of the selection
+ *     (never of memory safety).
+ *   - Limits: k <= 64, at most 64 constraint tokens per sentence, k*V < 2^31, V >= 1.
+ *
+ * Slot kinds: a slot is EMPTY when its score is -inf, FINISHED when it is live and its last token is
+ * eos_id, OPEN otherwise.  After dba_init (and dba_reset) slot 0 of every sentence is open with score 0
+ * and last token bos_id; slots 1..k-1 are empty.
+ */
+#ifndef DBA_H
+#define DBA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dba_handle dba_handle;
+
+typedef enum {
+    DBA_OK = 0,
+    DBA_ERR_INVALID_ARG = 1,   /* null pointer, bad size, malformed constraint table, bad token id      */
+    DBA_ERR_UNSUPPORTED = 2,   /* over a documented limit (k > 64, > 64 constraint tokens, k*V >= 2^31) */
+    DBA_ERR_STATE = 3,         /* step after max_steps, host-staging call without the staging flag     */
+    DBA_ERR_CUDA = 4,          /* a CUDA runtime call failed                                            */
+    DBA_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up (reported by dba_finalize)        */
+    DBA_ERR_WORKSPACE = 6      /* workspace too small or misaligned                                     */
+} dba_status;
+
+typedef enum { DBA_F32 = 0, DBA_BF16 = 1 } dba_dtype;
+
+enum {
+    DBA_FLAG_ADJUST_OFF   = 1u,  /* Section 5 (grid-beam-search simulation): no bank adjustment        */
+    DBA_FLAG_LENGTH_NORM  = 2u,  /* Section 4: dba_finalize ranks completed hypotheses by score/length  */
+    DBA_FLAG_HOST_STAGING = 4u   /* reserve workspace for dba_step_host                                 */
+};
+
+/*
+ * Problem statement (Section 3): a fixed beam size k and, per sentence, a set of word constraints (one
+ * token) and phrasal constraints (two or more contiguous tokens, met in order).  C_b, the number of
+ * constraints of sentence b, counts every token of every word and phrase.
+ * The constraint arrays are HOST memory, read during dba_init only; the caller keeps ownership.
+ */
+typedef struct {
+    int32_t B, k, V, max_steps;
+    int32_t pad_id, bos_id, eos_id;
+    int32_t logit_dtype;               /* dba_dtype */
+    uint32_t flags;
+    const int32_t* sent_phrase_off;    /* [B+1]  phrases of sentence b are [off[b], off[b+1])             */
+    const int32_t* phrase_tok_off;     /* [P+1]  tokens of phrase p are   [off[p], off[p+1]), non-empty   */
+    const int32_t* tok;                /* [sum]  token ids in [0, V), none of pad/bos/eos                 */
+} dba_config;
+
+/*
+ * Outputs of one step: the new beam, in decreasing score order (ties: lower back-pointer*V + token
+ * first), empty slots last.  Each array is [B*k]; any pointer may be NULL (that output is skipped).
+ * dba_step takes DEVICE pointers here, dba_step_host takes HOST pointers.
+ *   backptr   beam slot (0..k-1) of the previous beam this hypothesis extends (Algorithm 2: i of (i,j))
+ *   token     the token generated (Algorithm 2: j of (i,j)); pad_id for empty slots
+ *   score     cumulative log-probability (fp32); -inf for empty slots
+ *   bank      number of constraint tokens met (Section 3.2); -1 for empty slots
+ *   met_mask  bit j set = constraint token position j (phrases flattened in order) is marked met
+ *   active    position of the last met token of a begun, unfinished phrase, else -1
+ *   row_lse   log-sum-exp of the INPUT rows of this step (fp32; 0 for rows that were not open)
+ */
+typedef struct {
+    int32_t*  backptr;
+    int32_t*  token;
+    float*    score;
+    int32_t*  bank;
+    uint64_t* met_mask;
+    int32_t*  active;
+    float*    row_lse;
+} dba_step_out;
+
+/* Bytes of device workspace a handle for this configuration needs (256-byte aligned base). */
+dba_status dba_workspace_bytes(const dba_config* cfg, size_t* bytes);
+
+/*
+ * Validates cfg, flattens the constraint tables, copies them to the workspace and sets the initial
+ * beam (Algorithm 1, DECODER-INIT).  `cuda_stream` is a cudaStream_t (NULL = default stream); all later
+ * work of the handle is enqueued on it.  Synchronises the stream once before returning.
+ */
+dba_status dba_init(const dba_config* cfg, void* workspace_dev, size_t workspace_bytes,
+                    void* cuda_stream, dba_handle** out);
+
+/* Back to the initial beam and step 0, same constraints (enqueued; does not synchronise). */
+dba_status dba_reset(dba_handle* h);
+
+/*
+ * One timestep (Algorithm 2).  logits_dev: [B*k, V] of the configured dtype, element (r, w) at
+ * logits_dev[r*row_stride_elems + w]; row r must hold the model output for the hypothesis currently in
+ * beam slot r (the caller re-orders its decoder state by the previous step's backptr).
+ * Rows of empty and finished slots are not read.
+ *   Section 2 / 3.1  score(h, w) = fl32(fl32(x[h,w] - lse_h) + score_h); a finished slot only continues
+ *                    with eos_id at an unchanged score.
+ *   Section 3.3      score(h, eos_id) = -inf while slot h has unmet constraint tokens.
+ *   Section 3.1      candidates = the k best cells of the k x V matrix, every token that advances an
+ *                    open slot through its constraints, and every live slot's best token; each carries
+ *                    its updated constraint marks (a broken phrase is unwound).
+ *   Section 3.2      the k slots are divided over the C_b+1 banks (floor(k/(C_b+1)) each, the rest to
+ *                    the top bank; unfillable slots move to the nearest banks that can use them) and
+ *                    each bank keeps its best candidates.
+ * row_lse_in_dev (optional, [B*k] fp32): when non-NULL, the row normalisers are taken from it instead
+ * of being computed from the logits (e.g. all zeros when the rows are log-probabilities already); the
+ * computed values are still what out->row_lse reports.
+ * Returns DBA_ERR_STATE after max_steps steps.
+ */
+dba_status dba_step(dba_handle* h, const void* logits_dev, int64_t row_stride_elems,
+                    const float* row_lse_in_dev, const dba_step_out* out_dev);
+
+/*
+ * The same step with HOST buffers: copies the logits to a staging area in the workspace, runs the
+ * step, copies the requested outputs back and synchronises the stream.  Needs DBA_FLAG_HOST_STAGING.
+ * Pinned host memory makes the copies asynchronous with respect to the host until the final wait.
+ */
+dba_status dba_step_host(dba_handle* h, const void* logits_host, int64_t row_stride_elems,
+                         const dba_step_out* out_host);
+
+/*
+ * Section 3.3: per sentence the completed hypothesis (last token eos_id) with the highest score
+ * (score / length with DBA_FLAG_LENGTH_NORM, length counting the end token), lowest slot on ties; if
+ * none is completed, the best live slot of the highest occupied bank, flagged not completed.
+ * tokens_host [B, max_steps]: generated tokens up to and including the first eos_id (bos excluded),
+ * padded with pad_id;  len_host [B];  score_host [B];  flags_host [B], bit 0 = completed.
+ * Any pointer may be NULL.  Synchronises the stream.  Returns DBA_ERR_TIMEOUT / DBA_ERR_CUDA if a
+ * kernel of an earlier step recorded a problem in the device status word.
+ */
+dba_status dba_finalize(dba_handle* h, int32_t* tokens_host, int32_t* len_host, float* score_host,
+                        int32_t* flags_host);
+
+/* Number of kernels this handle has launched so far (for accounting in benchmarks). */
+uint64_t dba_launch_count(const dba_handle* h);
+
+/* Frees the handle (not the workspace). NULL is allowed. */
+void dba_destroy(dba_handle* h);
+
+const char* dba_status_string(dba_status s);
+
+/*
+ * The first kernel of the step on its own (Section 2's row normaliser plus the ARGMAX_K of
+ * Algorithm 1 restricted to single rows): for each of R rows of V logits, the log-sum-exp and the
+ * n_top largest entries in order (value descending, lower index first among equals).
+ *   row_lse_dev [R] fp32;  top_val_dev [R, n_top] fp32 (widened);  top_idx_dev [R, n_top] int32.
+ * If V < n_top the tail is filled with (-inf, -1).  scratch_dev must hold dba_row_scan_scratch_bytes.
+ * Enqueues on `cuda_stream`, does not synchronise.  n_top <= 66.
+ */
+dba_status dba_row_scan_scratch_bytes(int32_t R, int32_t V, int32_t n_top, int32_t logit_dtype, size_t* bytes);
+dba_status dba_row_scan(const void* logits_dev, int32_t logit_dtype, int32_t R, int32_t V,
+                        int64_t row_stride_elems, int32_t n_top, void* scratch_dev, size_t scratch_bytes,
+                        float* row_lse_dev, float* top_val_dev, int32_t* top_idx_dev, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DBA_H */

@@ -13,6 +13,7 @@
  * Where the paper is silent the reading taken is marked "READING" below.  Pin
  * status (what the CPU tests tie each function to, other than itself):
  *   orc_row_lse        pinned   closed forms (constant, two-value, geometric rows), shift invariance
+ *   orc_row_top        pinned   equals a stable descending sort of the row
  *   step at C = 0      pinned   equals Algorithm 1's ARGMAX_K over the k x V matrix (full sort)
  *   candidate set      pinned   brute force by predicate over every (h, w) cell on small V, k
  *   orc_add            pinned   hand traces of Section 3.1's unwinding text; substring semantics on
@@ -88,6 +89,27 @@ double orc_row_lse(const void *row, int dtype, int V)
     double s = 0.0;
     for (int w = 0; w < V; ++w) s += exp((double)widen(row, dtype, w) - m);
     return m + log(s);
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Algorithm 1, ARGMAX_K restricted to one row: the n largest entries in order, by taking the best
+ * remaining entry n times (value descending; READING: the lower index first among equal values).
+ * Fewer than n entries: the tail is (-inf, -1).
+ * ------------------------------------------------------------------------------------------ */
+void orc_row_top(const void *row, int dtype, int V, int n, float *val_out, int *idx_out)
+{
+    unsigned char *taken = (unsigned char *)calloc((size_t)V, 1);
+    for (int i = 0; i < n; ++i) {
+        int best = -1;
+        for (int w = 0; w < V; ++w) {
+            if (taken[w]) continue;
+            if (best < 0 || widen(row, dtype, w) > widen(row, dtype, best)) best = w;
+        }
+        if (best < 0) { val_out[i] = -INFINITY; idx_out[i] = -1; continue; }
+        taken[best] = 1;
+        val_out[i] = widen(row, dtype, best); idx_out[i] = best;
+    }
+    free(taken);
 }
 
 /* ------------------------------------------------------------------------------------------

@@ -38,6 +38,7 @@ def lib():
         i32p, f32p, u64p = C.POINTER(C.c_int32), C.POINTER(C.c_float), C.POINTER(C.c_uint64)
         L.orc_row_lse.restype = C.c_double
         L.orc_row_lse.argtypes = [C.c_void_p, C.c_int, C.c_int]
+        L.orc_row_top.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, f32p, i32p]
         L.orc_create.restype = C.c_void_p
         L.orc_create.argtypes = [C.c_int] * 6 + [C.c_uint, C.c_int, i32p, i32p]
         L.orc_destroy.argtypes = [C.c_void_p]
@@ -66,6 +67,16 @@ def row_lse(row: np.ndarray) -> float:
     dt = F32 if row.dtype == np.float32 else BF16
     assert row.dtype in (np.float32, np.uint16)
     return lib().orc_row_lse(row.ctypes.data, dt, row.size)
+
+
+def row_top(row: np.ndarray, n: int):
+    """The n largest entries of one row in order (value descending, lower index first)."""
+    row = np.ascontiguousarray(row)
+    dt = F32 if row.dtype == np.float32 else BF16
+    assert row.dtype in (np.float32, np.uint16)
+    val = np.zeros(n, np.float32); idx = np.zeros(n, np.int32)
+    lib().orc_row_top(row.ctypes.data, dt, row.size, n, _p(val, C.c_float), _p(idx, C.c_int32))
+    return val, idx
 
 
 def allocate(k: int, n, flags: int = 0) -> np.ndarray:

@@ -1,0 +1,215 @@
+// Allocation kernel (Section 3.2: ALLOCATE of Algorithm 2, then newBeam), one warp per sentence; plus the
+// small kernels that reset the beam and pick / trace back the final hypothesis (Section 3.3).
+#include "dba_device.cuh"
+#include "dba_internal.h"
+
+namespace dba {
+
+namespace {
+
+constexpr int kAllocWarps = 4;       // sentences per CTA
+constexpr int kBanks = kMaxC + 1;
+
+// Nearest bank above / below b whose bit is set in the 65-bit set (lo: banks 0..63, hi: bank 64); -1 if none.
+__device__ __forceinline__ int next_above(uint64_t lo, bool hi, int b) {
+    if (b < 63) {
+        const uint64_t m = lo & ~((2ull << b) - 1ull);
+        if (m) return __ffsll((long long)m) - 1;
+    }
+    return (hi && b < 64) ? 64 : -1;
+}
+__device__ __forceinline__ int next_below(uint64_t lo, int b) {
+    const uint64_t m = b >= 64 ? lo : (lo & ((1ull << b) - 1ull));
+    return m ? 63 - __clzll((long long)m) : -1;
+}
+
+__global__ void __launch_bounds__(kAllocWarps * 32)
+allocate_kernel(Dims d, const SentCons* __restrict__ cons, Beam cur, Beam nxt, const Cand* __restrict__ cand,
+                const int32_t* __restrict__ ncand, const int32_t* __restrict__ bank_count,
+                const float* __restrict__ row_lse, dba_step_out out, int32_t* __restrict__ hist_bp,
+                int32_t* __restrict__ hist_tok) {
+    __shared__ int s_n[kAllocWarps][kBanks];
+    __shared__ int s_alloc[kAllocWarps][kBanks];
+    __shared__ int s_off[kAllocWarps][kBanks];
+    __shared__ int s_sel[kAllocWarps][kMaxK];
+    __shared__ float s_score[kAllocWarps][kMaxK];
+    __shared__ int s_flat[kAllocWarps][kMaxK];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x * kAllocWarps + warp;
+    if (b >= d.B) return;
+    const int k = d.k, V = d.V;
+    const int C = cons[b].C;
+    int* n = s_n[warp]; int* alloc = s_alloc[warp]; int* off = s_off[warp]; int* sel = s_sel[warp];
+
+    // bank sizes; equal base share, remainder to the top bank C (Section 3.2)
+    const int share = k / (C + 1);
+    for (int q = lane; q <= C; q += 32) {
+        n[q] = bank_count[b * kBanks + q];
+        alloc[q] = share + (q == C ? k - share * (C + 1) : 0);
+    }
+    __syncwarp();
+    if (lane == 0) {
+        // exclusive offsets of the banks inside the bank-ordered candidate list
+        int acc = 0;
+        for (int q = 0; q <= C; ++q) { off[q] = acc; acc += n[q]; }
+        if (d.flags & DBA_FLAG_ADJUST_OFF) {
+            for (int q = 0; q <= C; ++q) alloc[q] = min(alloc[q], n[q]);
+        } else {
+            // Adjustment: every bank with more slots than candidates passes the surplus to the nearest
+            // banks that have more candidates than slots, the higher one first at equal distance.
+            uint64_t over_lo = 0, need_lo = 0; bool over_hi = false, need_hi = false;
+            for (int q = 0; q <= C; ++q) {
+                const bool ov = alloc[q] > n[q], nd = n[q] > alloc[q];
+                if (q < 64) { over_lo |= (uint64_t)ov << q; need_lo |= (uint64_t)nd << q; }
+                else { over_hi = ov; need_hi = nd; }
+            }
+            for (int q = 0; q <= C; ++q) {
+                const bool ov = q < 64 ? ((over_lo >> q) & 1ull) : over_hi;
+                if (!ov) continue;
+                int surplus = alloc[q] - n[q];
+                alloc[q] = n[q];
+                while (surplus > 0) {
+                    const int up = next_above(need_lo, need_hi, q);
+                    const int dn = next_below(need_lo, q);
+                    int r;
+                    if (up < 0 && dn < 0) break;
+                    if (up >= 0 && (dn < 0 || up - q <= q - dn)) r = up; else r = dn;
+                    const int g = min(surplus, n[r] - alloc[r]);
+                    alloc[r] += g; surplus -= g;
+                    if (alloc[r] == n[r]) { if (r < 64) need_lo &= ~(1ull << r); else need_hi = false; }
+                }
+            }
+        }
+        // the best alloc[q] candidates of every bank (they are ordered inside the bank already)
+        int ns = 0;
+        for (int q = 0; q <= C; ++q)
+            for (int i = 0; i < alloc[q]; ++i) sel[ns++] = off[q] + i;
+        off[0] = ns;   // reuse as the selected count
+    }
+    __syncwarp();
+    const int ns = off[0];
+    const Cand* cb = cand + (int64_t)b * d.max_cand;
+    for (int i = lane; i < ns; i += 32) { s_score[warp][i] = cb[sel[i]].score; s_flat[warp][i] = cb[sel[i]].flat; }
+    __syncwarp();
+    // new beam in decreasing score order, ties by lower flat index (Section 3.1), empty slots last
+    const int r0 = b * k;
+    for (int i = lane; i < k; i += 32) {
+        if (i < ns) {
+            const float si = s_score[warp][i]; const int fi = s_flat[warp][i];
+            int rank = 0;
+            for (int j = 0; j < ns; ++j) rank += cell_better(s_score[warp][j], s_flat[warp][j], si, fi);
+            const Cand c = cb[sel[i]];
+            const int h = fi / V, w = fi - h * V;
+            const int r = r0 + rank;
+            const int bank = __popcll(c.mask);
+            const int plen = cur.len[r0 + h];
+            const int len = cur.token[r0 + h] == d.eos_id ? plen : plen + 1;
+            nxt.score[r] = si; nxt.token[r] = w; nxt.mask[r] = c.mask; nxt.active[r] = c.active; nxt.len[r] = len;
+            nxt.bank[r] = bank; nxt.backptr[r] = h;
+            hist_bp[r] = h; hist_tok[r] = w;
+            if (out.backptr) out.backptr[r] = h;
+            if (out.token) out.token[r] = w;
+            if (out.score) out.score[r] = si;
+            if (out.bank) out.bank[r] = bank;
+            if (out.met_mask) out.met_mask[r] = c.mask;
+            if (out.active) out.active[r] = c.active;
+        }
+    }
+    for (int i = ns + lane; i < k; i += 32) {
+        const int r = r0 + i;
+        nxt.score[r] = neg_inf(); nxt.token[r] = d.pad_id; nxt.mask[r] = 0; nxt.active[r] = -1; nxt.len[r] = 0;
+        nxt.bank[r] = -1; nxt.backptr[r] = 0;
+        hist_bp[r] = 0; hist_tok[r] = d.pad_id;
+        if (out.backptr) out.backptr[r] = 0;
+        if (out.token) out.token[r] = d.pad_id;
+        if (out.score) out.score[r] = neg_inf();
+        if (out.bank) out.bank[r] = -1;
+        if (out.met_mask) out.met_mask[r] = 0;
+        if (out.active) out.active[r] = -1;
+    }
+    if (out.row_lse)
+        for (int i = lane; i < k; i += 32) out.row_lse[r0 + i] = row_lse[r0 + i];
+}
+
+// Algorithm 1, DECODER-INIT: slot 0 holds the start symbol at score 0, the other slots are empty.
+__global__ void reset_kernel(Dims d, Beam beam) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= d.R) return;
+    const bool first = (r % d.k) == 0;
+    beam.score[r] = first ? 0.f : neg_inf();
+    beam.token[r] = first ? d.bos_id : d.pad_id;
+    beam.mask[r] = 0; beam.active[r] = -1; beam.len[r] = 0; beam.bank[r] = first ? 0 : -1; beam.backptr[r] = 0;
+}
+
+// Section 3.3: the completed hypothesis with the highest score (Section 4: optionally divided by its
+// length); if none is completed, the best live slot of the highest occupied bank.  One thread per sentence.
+__global__ void finalize_kernel(Dims d, Beam beam, const int32_t* __restrict__ hist_bp,
+                                const int32_t* __restrict__ hist_tok, int steps, int max_steps,
+                                int32_t* __restrict__ tokens, int32_t* __restrict__ len_out,
+                                float* __restrict__ score_out, int32_t* __restrict__ flags_out) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= d.B) return;
+    const int k = d.k, r0 = b * k;
+    int pick = -1; float val = 0.f;
+    for (int h = 0; h < k; ++h) {
+        const float s = beam.score[r0 + h];
+        if (s == neg_inf() || beam.token[r0 + h] != d.eos_id) continue;
+        float v = s;
+        const int L = beam.len[r0 + h];
+        if ((d.flags & DBA_FLAG_LENGTH_NORM) && L > 0) v = __fdiv_rn(s, (float)L);
+        if (pick < 0 || v > val) { pick = h; val = v; }
+    }
+    const bool completed = pick >= 0;
+    if (!completed) {
+        int best_bank = -1;
+        for (int h = 0; h < k; ++h) {
+            const float s = beam.score[r0 + h];
+            if (s == neg_inf()) continue;
+            const int bk = __popcll(beam.mask[r0 + h]);
+            if (bk > best_bank || (bk == best_bank && s > val)) { best_bank = bk; pick = h; val = s; }
+        }
+    }
+    int32_t* out = tokens + (int64_t)b * max_steps;
+    for (int t = 0; t < max_steps; ++t) out[t] = d.pad_id;
+    flags_out[b] = completed ? 1 : 0;
+    score_out[b] = pick < 0 ? neg_inf() : val;
+    if (pick < 0 || steps == 0) { len_out[b] = 0; return; }
+    int slot = pick;
+    for (int t = steps - 1; t >= 0; --t) {        // walk the back-pointers, writing tokens in place
+        out[t] = hist_tok[(int64_t)t * d.R + r0 + slot];
+        slot = hist_bp[(int64_t)t * d.R + r0 + slot];
+    }
+    int n = 0;
+    while (n < steps) { ++n; if (out[n - 1] == d.eos_id) break; }
+    for (int t = n; t < steps; ++t) out[t] = d.pad_id;
+    len_out[b] = n;
+}
+
+}  // namespace
+
+cudaError_t launch_allocate(const Dims& d, const SentCons* cons, const Beam& cur, const Beam& next,
+                            const Cand* cand, const int32_t* ncand, const int32_t* bank_count,
+                            const float* row_lse, const dba_step_out& out, int32_t* hist_bp, int32_t* hist_tok,
+                            cudaStream_t st, int* launches) {
+    allocate_kernel<<<(d.B + kAllocWarps - 1) / kAllocWarps, kAllocWarps * 32, 0, st>>>(
+        d, cons, cur, next, cand, ncand, bank_count, row_lse, out, hist_bp, hist_tok);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reset(const Dims& d, const Beam& beam, cudaStream_t st, int* launches) {
+    reset_kernel<<<(d.R + 255) / 256, 256, 0, st>>>(d, beam);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_finalize(const Dims& d, const Beam& beam, const int32_t* hist_bp, const int32_t* hist_tok,
+                            int32_t steps, int32_t max_steps, int32_t* tokens, int32_t* len, float* score,
+                            int32_t* flags, cudaStream_t st, int* launches) {
+    finalize_kernel<<<(d.B + 127) / 128, 128, 0, st>>>(d, beam, hist_bp, hist_tok, steps, max_steps, tokens, len,
+                                                       score, flags);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace dba

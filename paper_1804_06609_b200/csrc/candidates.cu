@@ -1,0 +1,393 @@
+// Candidate kernel (Algorithm 2 up to the call of ALLOCATE; Section 3.1; Section 3.3's end-token rule).
+// One CTA per sentence.  Builds the candidate set from (1) the k best cells of the k x V score matrix,
+// (2) every token that advances an open hypothesis through its constraints and (3) every live
+// hypothesis' best token, updates the constraint marks of each candidate (unwinding a broken phrase),
+// removes duplicates, and hands the candidates over grouped by bank and ordered inside each bank.
+#include "dba_device.cuh"
+#include "dba_internal.h"
+
+namespace dba {
+
+namespace {
+
+constexpr int kCandThreads = 256;
+constexpr int kCandWarps = kCandThreads / 32;
+
+struct SortEnt {
+    uint64_t hi;   // bank << 32 | (~ordered score): ascending = bank ascending, score descending
+    uint32_t lo;   // flat index h*V + w, ascending
+    uint32_t id;   // position in the unsorted candidate arrays
+};
+
+struct Layout {   // byte offsets into dynamic shared memory
+    int cons, parent, lse, mask, active, kind, eos_ok, rt_score, rt_w, rt_n, rt_ptr, s1_h, s1_i, stage, merged,
+        tmp_score, tmp_w, c_score, c_flat, c_mask, c_active, bank_cnt, sort, total;
+    int n_sort;
+};
+
+__host__ __device__ inline int align_up(int x, int a) { return (x + a - 1) / a * a; }
+__host__ __device__ inline int next_pow2(int x) { int p = 32; while (p < x) p <<= 1; return p; }
+
+__host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand) {
+    Layout L;
+    int o = 0;
+    L.cons = o;      o = align_up(o + (int)sizeof(SentCons), 16);
+    L.mask = o;      o += 8 * k;
+    L.parent = o;    o += 4 * k;
+    L.lse = o;       o += 4 * k;
+    L.active = o;    o += 4 * k;
+    L.kind = o;      o += 4 * k;
+    L.eos_ok = o;    o += 4 * k;
+    L.rt_score = o;  o += 4 * k * k;
+    L.rt_w = o;      o += 4 * k * k;
+    L.rt_n = o;      o += 4 * k;
+    L.rt_ptr = o;    o += 4 * k;
+    L.s1_h = o;      o += 4 * k;
+    L.s1_i = o;      o += 4 * k;
+    o = align_up(o, 8);
+    L.stage = o;     o += 8 * kCandWarps * (S > 1 ? S * K1 : 0);
+    L.merged = o;    o += 8 * kCandWarps * K1;
+    L.tmp_score = o; o += 4 * kCandWarps * (k + 1);
+    L.tmp_w = o;     o += 4 * kCandWarps * (k + 1);
+    o = align_up(o, 8);
+    L.c_mask = o;    o += 8 * max_cand;
+    L.c_score = o;   o += 4 * max_cand;
+    L.c_flat = o;    o += 4 * max_cand;
+    L.c_active = o;  o += 4 * max_cand;
+    L.bank_cnt = o;  o += 4 * (kMaxC + 1);
+    o = align_up(o, 16);
+    L.n_sort = next_pow2(max_cand);
+    L.sort = o;      o += (int)sizeof(SortEnt) * L.n_sort;
+    L.total = o;
+    return L;
+}
+
+// constraints[h].add(w): Section 3.1 (last paragraph).  Continue the begun phrase if w is its next token;
+// otherwise reset that phrase's marks and let w open the first wholly unmet word/phrase it matches.
+__device__ __forceinline__ void cons_add(const SentCons& sc, uint64_t& mask, int& active, int w) {
+    if (active >= 0) {
+        const int n = active + 1;
+        if (w == sc.ctok[n]) {
+            mask |= 1ull << n;
+            active = ((sc.last_mask >> n) & 1ull) ? -1 : n;
+            return;
+        }
+        const int p0 = sc.pstart[active];
+        const uint64_t span = ((2ull << active) - 1ull) & ~((1ull << p0) - 1ull);   // bits p0..active
+        mask &= ~span;
+        active = -1;
+    }
+    uint64_t open = sc.first_mask & ~mask;
+    while (open) {
+        const int j = __ffsll((long long)open) - 1;
+        if (sc.ctok[j] == w) {
+            mask |= 1ull << j;
+            active = ((sc.last_mask >> j) & 1ull) ? -1 : j;
+            return;
+        }
+        open &= open - 1;
+    }
+}
+
+__global__ void __launch_bounds__(kCandThreads)
+candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const SentCons* __restrict__ cons,
+                  Beam cur, ScanOut part, const float* __restrict__ lse_in, float* __restrict__ row_lse,
+                  Cand* __restrict__ cand_out, int32_t* __restrict__ ncand_out, int32_t* __restrict__ bank_count,
+                  uint32_t* __restrict__ status) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int k = d.k, V = d.V, K1 = d.K1, S = d.S;
+    const Layout L = make_layout(k, K1, S, d.max_cand);
+    SentCons& sc = *reinterpret_cast<SentCons*>(smem + L.cons);
+    uint64_t* s_mask = reinterpret_cast<uint64_t*>(smem + L.mask);
+    float* s_parent = reinterpret_cast<float*>(smem + L.parent);
+    float* s_lse = reinterpret_cast<float*>(smem + L.lse);
+    int* s_active = reinterpret_cast<int*>(smem + L.active);
+    int* s_kind = reinterpret_cast<int*>(smem + L.kind);      // 0 empty, 1 open, 2 finished
+    int* s_eos_ok = reinterpret_cast<int*>(smem + L.eos_ok);
+    float* rt_score = reinterpret_cast<float*>(smem + L.rt_score);
+    int* rt_w = reinterpret_cast<int*>(smem + L.rt_w);
+    int* rt_n = reinterpret_cast<int*>(smem + L.rt_n);
+    int* rt_ptr = reinterpret_cast<int*>(smem + L.rt_ptr);
+    int* s1_h = reinterpret_cast<int*>(smem + L.s1_h);
+    int* s1_i = reinterpret_cast<int*>(smem + L.s1_i);
+    float* c_score = reinterpret_cast<float*>(smem + L.c_score);
+    int* c_flat = reinterpret_cast<int*>(smem + L.c_flat);
+    uint64_t* c_mask = reinterpret_cast<uint64_t*>(smem + L.c_mask);
+    int* c_active = reinterpret_cast<int*>(smem + L.c_active);
+    int* bank_cnt = reinterpret_cast<int*>(smem + L.bank_cnt);
+    SortEnt* ent = reinterpret_cast<SortEnt*>(smem + L.sort);
+    __shared__ int s_ncand, s_ns1;
+
+    const int b = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int r0 = b * k;
+
+    // ---- load the sentence: constraint table and beam state --------------------------------------------
+    {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(cons + b);
+        uint32_t* dst = reinterpret_cast<uint32_t*>(&sc);
+        for (int i = tid; i < (int)(sizeof(SentCons) / 4); i += kCandThreads) dst[i] = src[i];
+    }
+    if (tid < k) {
+        const float ps = cur.score[r0 + tid];
+        const int tk = cur.token[r0 + tid];
+        s_parent[tid] = ps;
+        s_mask[tid] = cur.mask[r0 + tid];
+        s_active[tid] = cur.active[r0 + tid];
+        s_kind[tid] = ps == neg_inf() ? 0 : (tk == d.eos_id ? 2 : 1);
+        rt_ptr[tid] = 0;
+        rt_n[tid] = 0;
+    }
+    if (tid <= kMaxC) bank_cnt[tid] = 0;
+    if (tid == 0) { s_ncand = 0; s_ns1 = 0; }
+    __syncthreads();
+    const int C = sc.C;
+    if (tid < k) s_eos_ok[tid] = __popcll(s_mask[tid]) >= C;   // Section 3.3: end token only once all are met
+    __syncthreads();
+
+    // ---- phase A: per row, the k best cells in (score desc, token asc) order ------------------------------
+    uint64_t* stage = reinterpret_cast<uint64_t*>(smem + L.stage) + warp * (S > 1 ? S * K1 : 0);
+    uint64_t* merged = reinterpret_cast<uint64_t*>(smem + L.merged) + warp * K1;
+    float* tmp_score = reinterpret_cast<float*>(smem + L.tmp_score) + warp * (k + 1);
+    int* tmp_w = reinterpret_cast<int*>(smem + L.tmp_w) + warp * (k + 1);
+    const unsigned lt_mask = (1u << lane) - 1u;
+
+    for (int h = warp; h < k; h += kCandWarps) {
+        const int r = r0 + h;
+        const int kind = s_kind[h];
+        if (kind == 0) { if (lane == 0) { row_lse[r] = 0.f; s_lse[h] = 0.f; } continue; }
+        if (kind == 2) {                      // finished: repeats the end token at an unchanged score
+            if (lane == 0) { rt_n[h] = 1; rt_score[h * k] = s_parent[h]; rt_w[h * k] = d.eos_id; row_lse[r] = 0.f; s_lse[h] = 0.f; }
+            continue;
+        }
+        // row normaliser from the segment partials (fixed order)
+        float lse;
+        {
+            float M = neg_inf();
+            for (int g = 0; g < S; ++g) M = fmaxf(M, part.m[r * S + g]);
+            float sum = 0.f;
+            if (M != neg_inf())
+                for (int g = 0; g < S; ++g) {
+                    const float mg = part.m[r * S + g];
+                    if (mg != neg_inf()) sum += part.s[r * S + g] * expf(mg - M);
+                }
+            lse = M == neg_inf() ? neg_inf() : M + logf(sum);
+        }
+        if (lane == 0) row_lse[r] = lse;
+        if (lse_in) lse = lse_in[r];
+        if (lane == 0) s_lse[h] = lse;
+        const float parent = s_parent[h];
+        const bool eos_ok = s_eos_ok[h] != 0;
+
+        // the row's K1 largest raw logits, merged over segments, as keys in `merged`
+        if (S == 1) {
+            for (int e = lane; e < K1; e += 32) {
+                const int ix = part.top_idx[(int64_t)r * K1 + e];
+                merged[e] = ix >= 0 ? row_key(part.top_val[(int64_t)r * K1 + e], ix) : 0ull;
+            }
+        } else {
+            const int n = S * K1;
+            for (int e = lane; e < K1; e += 32) merged[e] = 0ull;
+            for (int e = lane; e < n; e += 32) {
+                const int ix = part.top_idx[(int64_t)r * n + e];
+                stage[e] = ix >= 0 ? row_key(part.top_val[(int64_t)r * n + e], ix) : 0ull;
+            }
+            __syncwarp();
+            for (int e = lane; e < n; e += 32) {
+                const uint64_t key = stage[e];
+                if (!key) continue;
+                int rank = 0;
+                for (int j = 0; j < n; ++j) rank += stage[j] > key;
+                if (rank < K1) merged[rank] = key;
+            }
+        }
+        __syncwarp();
+
+        // scores of the entries that may be generated, in list order; keep k plus one sentinel
+        int total_valid = 0;
+        for (int e0 = 0; e0 < K1; e0 += 32) {
+            const int e = e0 + lane;
+            bool valid = false; float scv = neg_inf(); int w = -1;
+            if (e < K1) {
+                const uint64_t key = merged[e];
+                if (key) {
+                    const float x = row_key_val(key);
+                    w = row_key_idx(key);
+                    valid = x != neg_inf() && !(w == d.eos_id && !eos_ok) && lse != neg_inf();
+                    if (valid) scv = cell_score(x, lse, parent);
+                }
+            }
+            const unsigned bal = __ballot_sync(kFullMask, valid);
+            const int pos = total_valid + __popc(bal & lt_mask);
+            if (valid && pos <= k) { tmp_score[pos] = scv; tmp_w[pos] = w; }
+            total_valid += __popc(bal);
+        }
+        __syncwarp();
+        int nrow = min(total_valid, k);
+        // Distinct logits can round to one score.  If that happens across the cut between the k-th and
+        // the (k+1)-th entry, cells outside the list may tie with the k-th and precede it by index:
+        // rescan the whole row for the cells with exactly that score, lowest token ids first.
+        if (total_valid > k && tmp_score[k] == tmp_score[k - 1]) {
+            const float sb = tmp_score[k - 1];
+            int g = 0;
+            while (g < k && tmp_score[g] > sb) ++g;
+            const int need = k - g;
+            int found = 0;
+            __syncwarp();
+            for (int base = 0; base < V && found < need; base += 32) {
+                const int w = base + lane;
+                bool hit = false;
+                if (w < V) {
+                    const float x = load_logit_dyn(logits, d.dtype, (int64_t)r * stride + w);
+                    hit = x != neg_inf() && !(w == d.eos_id && !eos_ok) && cell_score(x, lse, parent) == sb;
+                }
+                const unsigned bal = __ballot_sync(kFullMask, hit);
+                const int pos = found + __popc(bal & lt_mask);
+                if (hit && pos < need) { tmp_score[g + pos] = sb; tmp_w[g + pos] = w; }
+                found += __popc(bal);
+            }
+            __syncwarp();
+        }
+        // order by (score desc, token asc) and publish
+        for (int i = lane; i < nrow; i += 32) {
+            const float si = tmp_score[i]; const int wi = tmp_w[i];
+            int rank = 0;
+            for (int j = 0; j < nrow; ++j) rank += cell_better(tmp_score[j], tmp_w[j], si, wi);
+            rt_score[h * k + rank] = si; rt_w[h * k + rank] = wi;
+        }
+        if (lane == 0) rt_n[h] = nrow;
+        __syncwarp();
+    }
+    __syncthreads();
+
+    // ---- phase B (source 1): the k best cells of the whole matrix, by a k-round tournament of row heads ----
+    if (warp == 0) {
+        int ns1 = 0;
+        for (int round = 0; round < k; ++round) {
+            float bs = neg_inf(); int bf = 0x7fffffff; int bh = -1;
+            for (int h = lane; h < k; h += 32) {
+                const int p = rt_ptr[h];
+                if (p < rt_n[h]) {
+                    const float s = rt_score[h * k + p]; const int f = h * V + rt_w[h * k + p];
+                    if (bh < 0 || cell_better(s, f, bs, bf)) { bs = s; bf = f; bh = h; }
+                }
+            }
+#pragma unroll
+            for (int o = 16; o; o >>= 1) {
+                const float os = __shfl_xor_sync(kFullMask, bs, o);
+                const int of = __shfl_xor_sync(kFullMask, bf, o);
+                const int oh = __shfl_xor_sync(kFullMask, bh, o);
+                if (oh >= 0 && (bh < 0 || cell_better(os, of, bs, bf))) { bs = os; bf = of; bh = oh; }
+            }
+            if (bh < 0) break;
+            if (lane == 0) { s1_h[ns1] = bh; s1_i[ns1] = rt_ptr[bh]; rt_ptr[bh] += 1; }
+            ++ns1;
+            __syncwarp();
+        }
+        if (lane == 0) s_ns1 = ns1;
+    }
+    __syncthreads();
+
+    // ---- sources 1 and 3 with their updated constraint marks; cells that advance a hypothesis through
+    //      its constraints are left to source 2, which lists every such cell (no duplicates arise) ----------
+    const int ns1 = s_ns1;
+    for (int t = tid; t < 2 * k; t += kCandThreads) {
+        int h, i;
+        if (t < k) { if (t >= ns1) continue; h = s1_h[t]; i = s1_i[t]; }
+        else { h = t - k; i = 0; if (rt_n[h] == 0 || rt_ptr[h] > 0) continue; }   // best cell already in source 1
+        const int w = rt_w[h * k + i];
+        uint64_t m = s_mask[h]; int a = s_active[h];
+        if (s_kind[h] == 1) {
+            const int before = __popcll(m);
+            cons_add(sc, m, a, w);
+            if (__popcll(m) == before + 1) continue;
+        }
+        const int slot = atomicAdd(&s_ncand, 1);
+        if (slot < d.max_cand) {
+            c_score[slot] = rt_score[h * k + i]; c_flat[slot] = h * V + w; c_mask[slot] = m; c_active[slot] = a;
+            atomicAdd(&bank_cnt[__popcll(m)], 1);
+        }
+    }
+    // ---- source 2: for every open hypothesis the tokens that raise its met count by one -------------------
+    for (int t = tid; t < k * kMaxC; t += kCandThreads) {
+        const int h = t >> 6, j = t & 63;
+        if (j >= C || s_kind[h] != 1) continue;
+        const uint64_t m = s_mask[h]; const int a = s_active[h];
+        if (a >= 0) { if (j != a + 1) continue; }
+        else {
+            if (!((sc.first_mask >> j) & 1ull) || ((m >> j) & 1ull)) continue;
+            bool dup = false;                              // same token opens an earlier unmet phrase
+            uint64_t earlier = sc.first_mask & ~m & ((1ull << j) - 1ull);
+            while (earlier) { const int q = __ffsll((long long)earlier) - 1; dup |= sc.ctok[q] == sc.ctok[j]; earlier &= earlier - 1; }
+            if (dup) continue;
+        }
+        const int w = sc.ctok[j];
+        const float x = load_logit_dyn(logits, d.dtype, (int64_t)(r0 + h) * stride + w);
+        const float lse = s_lse[h];
+        if (x == neg_inf() || lse == neg_inf()) continue;
+        const int slot = atomicAdd(&s_ncand, 1);
+        if (slot < d.max_cand) {
+            const uint64_t m2 = m | (1ull << j);
+            c_score[slot] = cell_score(x, lse, s_parent[h]); c_flat[slot] = h * V + w; c_mask[slot] = m2;
+            c_active[slot] = ((sc.last_mask >> j) & 1ull) ? -1 : j;
+            atomicAdd(&bank_cnt[__popcll(m2)], 1);
+        }
+    }
+    __syncthreads();
+    int n = s_ncand;
+    if (n > d.max_cand) { if (tid == 0) atomicOr(status, kStatusOverflow); n = d.max_cand; }
+
+    // ---- group by bank, order inside each bank (Section 3.1): bitonic sort on (bank, score desc, flat asc) --
+    int n_sort = 32;
+    while (n_sort < n) n_sort <<= 1;
+    for (int i = tid; i < n_sort; i += kCandThreads) {
+        SortEnt e;
+        if (i < n) {
+            e.hi = ((uint64_t)__popcll(c_mask[i]) << 32) | (uint32_t)(0xffffffffu - ord32(c_score[i]));
+            e.lo = (uint32_t)c_flat[i]; e.id = (uint32_t)i;
+        } else { e.hi = ~0ull; e.lo = 0xffffffffu; e.id = 0; }
+        ent[i] = e;
+    }
+    __syncthreads();
+    for (int size = 2; size <= n_sort; size <<= 1) {
+        for (int str = size >> 1; str > 0; str >>= 1) {
+            for (int t = tid; t < n_sort / 2; t += kCandThreads) {
+                const int pos = 2 * t - (t & (str - 1));
+                SortEnt a = ent[pos], c = ent[pos + str];
+                const bool gt = a.hi > c.hi || (a.hi == c.hi && a.lo > c.lo);
+                const bool up = (pos & size) == 0;
+                if (gt == up) { ent[pos] = c; ent[pos + str] = a; }
+            }
+            __syncthreads();
+        }
+    }
+    for (int i = tid; i < n; i += kCandThreads) {
+        const int id = ent[i].id;
+        Cand c; c.score = c_score[id]; c.flat = c_flat[id]; c.mask = c_mask[id]; c.active = c_active[id]; c.pad_ = 0;
+        cand_out[(int64_t)b * d.max_cand + i] = c;
+    }
+    if (tid <= kMaxC) bank_count[b * (kMaxC + 1) + tid] = bank_cnt[tid];
+    if (tid == 0) ncand_out[b] = n;
+}
+
+}  // namespace
+
+size_t candidates_smem_bytes(const Dims& d) { return (size_t)make_layout(d.k, d.K1, d.S, d.max_cand).total; }
+
+cudaError_t configure_candidates(const Dims& d) {
+    return cudaFuncSetAttribute(candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)candidates_smem_bytes(d));
+}
+
+cudaError_t launch_candidates(const void* logits, int64_t stride, const Dims& d, const SentCons* cons,
+                              const Beam& cur, const ScanOut& part, const float* lse_in, float* row_lse,
+                              Cand* cand, int32_t* ncand, int32_t* bank_count, uint32_t* status,
+                              cudaStream_t st, int* launches) {
+    const size_t smem = candidates_smem_bytes(d);
+    candidates_kernel<<<d.B, kCandThreads, smem, st>>>(logits, stride, d, cons, cur, part, lse_in, row_lse, cand,
+                                                      ncand, bank_count, status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace dba

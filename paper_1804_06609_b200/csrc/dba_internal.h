@@ -1,0 +1,97 @@
+// Internal declarations shared by the translation units of libdba (not part of the public ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dba.h"
+
+namespace dba {
+
+constexpr int kMaxK = 64;          // beam size limit
+constexpr int kMaxC = 64;          // constraint tokens per sentence (one bit each in a 64-bit mask)
+constexpr int kMaxTop = kMaxK + 2; // entries kept per row: k, one for a masked end token, one sentinel
+constexpr int kMaxSeg = 8;         // row segments scanned by different CTAs
+
+// device status word bits (sticky; read by dba_finalize)
+constexpr uint32_t kStatusTimeout = 1u;    // a bounded wait on an mbarrier gave up
+constexpr uint32_t kStatusOverflow = 2u;   // an internal list ran out of room (results of that step invalid)
+
+// Per-sentence constraint table, phrases flattened to token positions 0..C-1 (Section 3 of the paper:
+// the constraint count is the total number of tokens over all words and phrases).
+struct SentCons {
+    int32_t C;
+    int32_t n_phrases;
+    uint64_t first_mask;   // bit j: position j opens its word/phrase
+    uint64_t last_mask;    // bit j: position j closes its word/phrase
+    int32_t ctok[kMaxC];
+    uint8_t pstart[kMaxC]; // first position of the phrase position j belongs to
+};
+
+// One beam (all sentences): arrays of R = B*k entries.
+struct Beam {
+    float* score;
+    int32_t* token;
+    uint64_t* mask;
+    int32_t* active;
+    int32_t* len;
+    int32_t* bank;
+    int32_t* backptr;
+};
+
+// One candidate as handed from the candidate kernel to the allocation kernel.
+struct Cand {
+    float score;
+    int32_t flat;     // h*V + w
+    uint64_t mask;    // constraint marks after generating w
+    int32_t active;
+    int32_t pad_;
+};
+
+struct Dims {
+    int32_t B, k, V, R;
+    int32_t K1;        // entries kept per row segment by the scan kernel (k + 2, capped by the segment)
+    int32_t S;         // segments per row
+    int32_t seg_len;   // elements per segment (multiple of the scan kernel's chunk)
+    int32_t max_cand;  // candidate capacity per sentence
+    int32_t pad_id, bos_id, eos_id;
+    int32_t dtype;
+    uint32_t flags;
+};
+
+// Partial results of the row scan, one entry per (row, segment).
+struct ScanOut {
+    float* m;          // [R*S] reference maximum of the segment (-inf if it holds no finite value)
+    float* s;          // [R*S] sum of exp(x - m)
+    float* top_val;    // [R*S*K1] values, descending (ties: lower index first); (-inf, -1) padded
+    int32_t* top_idx;  // [R*S*K1] column within the row
+};
+
+// --- launchers (each enqueues on `st` and returns the CUDA error of the launch) ----------------------
+// `open_score` / `open_token` (may be null): rows whose slot is empty (score -inf) or finished
+// (token == eos) are skipped.
+cudaError_t launch_row_scan(const void* logits, int64_t stride, const Dims& d, const float* open_score,
+                            const int32_t* open_token, const ScanOut& out, uint32_t* status,
+                            cudaStream_t st, int* launches);
+cudaError_t launch_row_merge(const Dims& d, const ScanOut& part, int n_top, float* row_lse, float* top_val,
+                             int32_t* top_idx, cudaStream_t st, int* launches);
+cudaError_t launch_candidates(const void* logits, int64_t stride, const Dims& d, const SentCons* cons,
+                              const Beam& cur, const ScanOut& part, const float* lse_in, float* row_lse,
+                              Cand* cand, int32_t* ncand, int32_t* bank_count, uint32_t* status,
+                              cudaStream_t st, int* launches);
+cudaError_t launch_allocate(const Dims& d, const SentCons* cons, const Beam& cur, const Beam& next,
+                            const Cand* cand, const int32_t* ncand, const int32_t* bank_count,
+                            const float* row_lse, const dba_step_out& out, int32_t* hist_bp, int32_t* hist_tok,
+                            cudaStream_t st, int* launches);
+cudaError_t launch_reset(const Dims& d, const Beam& beam, cudaStream_t st, int* launches);
+cudaError_t launch_finalize(const Dims& d, const Beam& beam, const int32_t* hist_bp, const int32_t* hist_tok,
+                            int32_t steps, int32_t max_steps, int32_t* tokens, int32_t* len, float* score,
+                            int32_t* flags, cudaStream_t st, int* launches);
+
+size_t candidates_smem_bytes(const Dims& d);
+// Opts the candidate kernel in to the dynamic shared memory it needs on the current device.
+cudaError_t configure_candidates(const Dims& d);
+
+// Chooses S and seg_len for a row of V elements when R rows are scanned (fills d.S, d.seg_len, d.K1).
+void plan_segments(Dims& d, int sm_count);
+
+}  // namespace dba

@@ -1,0 +1,160 @@
+// Row scan: per (row, segment) the reference maximum, sum of exponentials and the K1 largest entries.
+// This file holds the generic kernel (any alignment, plain loads) and the stand-alone merge kernel.
+#include "dba_device.cuh"
+#include "dba_internal.h"
+
+namespace dba {
+
+namespace {
+
+constexpr int kScanThreads = 256;
+
+// Deterministic block reductions over kScanThreads threads (fixed tree, result broadcast to all).
+__device__ float block_max(float v, float* sm) {
+    v = warp_max(v);
+    if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = sm[0];
+    for (int i = 1; i < kScanThreads / 32; ++i) r = fmaxf(r, sm[i]);
+    __syncthreads();
+    return r;
+}
+__device__ float block_sum(float v, float* sm) {
+    v = warp_sum(v);
+    if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = sm[0];
+    for (int i = 1; i < kScanThreads / 32; ++i) r += sm[i];
+    __syncthreads();
+    return r;
+}
+__device__ uint64_t block_max_u64(uint64_t v, uint64_t* sm) {
+    v = warp_max_u64(v);
+    if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = v;
+    __syncthreads();
+    uint64_t r = sm[0];
+    for (int i = 1; i < kScanThreads / 32; ++i) r = sm[i] > r ? sm[i] : r;
+    __syncthreads();
+    return r;
+}
+
+// Generic scan: one CTA per (row, segment); K1 + 2 passes over the segment (it stays in L2).
+template <typename T>
+__global__ void __launch_bounds__(kScanThreads)
+row_scan_generic_kernel(const T* __restrict__ logits, int64_t stride, int V, int S, int seg_len, int K1,
+                        int eos, const float* __restrict__ open_score, const int32_t* __restrict__ open_token,
+                        float* __restrict__ part_m, float* __restrict__ part_s,
+                        float* __restrict__ top_val, int32_t* __restrict__ top_idx) {
+    __shared__ float smf[kScanThreads / 32];
+    __shared__ uint64_t smu[kScanThreads / 32];
+    const int item = blockIdx.x;
+    const int r = item / S, g = item - r * S;
+    if (open_score) {
+        if (open_score[r] == neg_inf() || open_token[r] == eos) return;   // empty or finished slot
+    }
+    const int lo = g * seg_len;
+    const int hi = min(V, lo + seg_len);
+    const T* row = logits + (int64_t)r * stride;
+
+    float m = neg_inf();
+    for (int w = lo + threadIdx.x; w < hi; w += kScanThreads) m = fmaxf(m, load_logit<T>(row + w));
+    m = block_max(m, smf);
+    float s = 0.f;
+    if (m != neg_inf())
+        for (int w = lo + threadIdx.x; w < hi; w += kScanThreads) s += expf(load_logit<T>(row + w) - m);
+    s = block_sum(s, smf);
+    if (threadIdx.x == 0) { part_m[item] = m; part_s[item] = s; }
+
+    uint64_t prev = ~0ull;
+    for (int i = 0; i < K1; ++i) {
+        uint64_t best = 0;
+        for (int w = lo + threadIdx.x; w < hi; w += kScanThreads) {
+            uint64_t key = row_key(load_logit<T>(row + w), w);
+            if (key < prev && key > best) best = key;
+        }
+        best = block_max_u64(best, smu);
+        if (threadIdx.x == 0) {
+            top_val[(int64_t)item * K1 + i] = best ? row_key_val(best) : neg_inf();
+            top_idx[(int64_t)item * K1 + i] = best ? row_key_idx(best) : -1;
+        }
+        prev = best ? best : 0;   // once exhausted, nothing is below key 0
+    }
+}
+
+// Stand-alone merge of the S segment results of each row: log-sum-exp and the n_top best entries.
+// One warp per row.
+__global__ void row_merge_kernel(int R, int S, int K1, int n_top, const float* __restrict__ part_m,
+                                 const float* __restrict__ part_s, const float* __restrict__ pv,
+                                 const int32_t* __restrict__ pi, float* __restrict__ row_lse,
+                                 float* __restrict__ top_val, int32_t* __restrict__ top_idx) {
+    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (r >= R) return;
+    if (lane == 0) {
+        float M = neg_inf();
+        for (int g = 0; g < S; ++g) M = fmaxf(M, part_m[r * S + g]);
+        float sum = 0.f;
+        if (M != neg_inf())
+            for (int g = 0; g < S; ++g)
+                if (part_m[r * S + g] != neg_inf()) sum += part_s[r * S + g] * expf(part_m[r * S + g] - M);
+        row_lse[r] = M == neg_inf() ? neg_inf() : M + logf(sum);
+    }
+    const int n = S * K1;
+    const float* v = pv + (int64_t)r * n;
+    const int32_t* ix = pi + (int64_t)r * n;
+    for (int e = lane; e < n_top; e += 32) { top_val[(int64_t)r * n_top + e] = neg_inf(); top_idx[(int64_t)r * n_top + e] = -1; }
+    __syncwarp();
+    for (int e = lane; e < n; e += 32) {
+        if (ix[e] < 0) continue;
+        uint64_t key = row_key(v[e], ix[e]);
+        int rank = 0;
+        for (int j = 0; j < n; ++j)
+            if (ix[j] >= 0 && row_key(v[j], ix[j]) > key) ++rank;
+        if (rank < n_top) { top_val[(int64_t)r * n_top + rank] = v[e]; top_idx[(int64_t)r * n_top + rank] = ix[e]; }
+    }
+}
+
+}  // namespace
+
+void plan_segments(Dims& d, int sm_count) {
+    // Enough (row, segment) items to occupy every SM a few times over, segments of at least 4096
+    // elements, at most kMaxSeg per row; segment length a multiple of 2048 elements.
+    int S = 1;
+    const int want = 4 * sm_count;
+    while (S < kMaxSeg && d.R * S < want && (d.V + 2 * S - 1) / (2 * S) >= 4096) S *= 2;
+    int seg = (d.V + S - 1) / S;
+    seg = (seg + 2047) / 2048 * 2048;
+    S = (d.V + seg - 1) / seg;
+    d.S = S;
+    d.seg_len = seg;
+    d.K1 = d.k + 2;
+}
+
+cudaError_t launch_row_scan(const void* logits, int64_t stride, const Dims& d, const float* open_score,
+                            const int32_t* open_token, const ScanOut& out, uint32_t* status,
+                            cudaStream_t st, int* launches) {
+    (void)status;
+    const int items = d.R * d.S;
+    if (d.dtype == DBA_F32)
+        row_scan_generic_kernel<float><<<items, kScanThreads, 0, st>>>(
+            (const float*)logits, stride, d.V, d.S, d.seg_len, d.K1, d.eos_id, open_score, open_token, out.m,
+            out.s, out.top_val, out.top_idx);
+    else
+        row_scan_generic_kernel<__nv_bfloat16><<<items, kScanThreads, 0, st>>>(
+            (const __nv_bfloat16*)logits, stride, d.V, d.S, d.seg_len, d.K1, d.eos_id, open_score, open_token,
+            out.m, out.s, out.top_val, out.top_idx);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_row_merge(const Dims& d, const ScanOut& part, int n_top, float* row_lse, float* top_val,
+                             int32_t* top_idx, cudaStream_t st, int* launches) {
+    const int warps = 4;
+    row_merge_kernel<<<(d.R + warps - 1) / warps, warps * 32, 0, st>>>(d.R, d.S, d.K1, n_top, part.m, part.s,
+                                                                      part.top_val, part.top_idx, row_lse,
+                                                                      top_val, top_idx);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace dba

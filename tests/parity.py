@@ -1,0 +1,87 @@
+"""Helpers of the GPU parity tests: run the oracle and the CUDA library side by side on one workload."""
+from __future__ import annotations
+
+import numpy as np
+
+from oracle import dba_oracle as O
+from synth_inputs import LogitStream
+
+BEAM_FIELDS = ("backptr", "token", "bank", "met_mask", "active")
+
+
+def torch_dtype(wl):
+    import torch
+    return torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+
+
+def to_device_logits(x_np, wl, device="cuda:0"):
+    """numpy logits (float32, or uint16 bf16 bits) -> CUDA tensor of the workload's dtype, same bits."""
+    import torch
+    t = torch.from_numpy(x_np.view(np.int16) if x_np.dtype == np.uint16 else x_np).to(device)
+    return t.view(torch.bfloat16) if x_np.dtype == np.uint16 else t
+
+
+def to_host_logits(x_dev):
+    """CUDA logits -> numpy (float32, or uint16 bits for bf16), same bits."""
+    import torch
+    if x_dev.dtype == torch.bfloat16:
+        return x_dev.view(torch.int16).cpu().numpy().view(np.uint16)
+    return x_dev.cpu().numpy()
+
+
+def gpu_beam(out):
+    d = {f: out[f].cpu().numpy() for f in ("backptr", "token", "score", "bank", "active", "row_lse")}
+    d["met_mask"] = out["met_mask"].cpu().numpy().view(np.uint64)
+    return d
+
+
+def assert_beam_equal(got, want, where, fields=BEAM_FIELDS + ("score",)):
+    """Bit-exact comparison of a GPU beam with the oracle's; reports the first differing (sentence row, field)."""
+    for f in fields:
+        a, b = got[f], want[f]
+        if f == "score":
+            same = (a == b) | (np.isinf(a) & np.isinf(b))
+        else:
+            same = a == b
+        if not same.all():
+            r = int(np.nonzero(~same)[0][0])
+            raise AssertionError(f"{where}: field {f} differs first at row {r}: gpu {a[r]} oracle {b[r]}\n"
+                                 f"gpu    {({g: got[g][r] for g in fields})}\noracle {({g: want[g][r] for g in fields})}")
+
+
+def lockstep(wl, stepper, steps=None, threads=8, gpu_gen=None, lse_tol=1e-5, flags=0):
+    """Closed loop with the oracle's row normalisers handed to the CUDA step (the direction oracle -> GPU),
+    so that both rank the same fp32 score matrix: every selection output must then match bit for bit at
+    every step, and the normalisers the GPU computes itself must agree within lse_tol."""
+    import torch
+    steps = wl.steps if steps is None else steps
+    orc = O.Batch(wl.k, wl.V, steps, wl.constraints, flags=flags & 3, threads=threads)
+    host_gen = LogitStream(wl) if gpu_gen is None else None
+    worst = 0.0
+    for t in range(steps):
+        ob = orc.beam()
+        if gpu_gen is not None:      # generate on the device from the ORACLE's state, copy back for the oracle
+            x_dev = gpu_gen.step_logits(t, torch.from_numpy(ob["token"]).cuda(),
+                                        torch.from_numpy(ob["met_mask"].view(np.int64)).cuda())
+            x_np = to_host_logits(x_dev)
+        else:
+            x_np = host_gen.step_logits(t, ob["token"], ob["met_mask"])
+            x_dev = to_device_logits(x_np, wl)
+        open_rows = np.isfinite(ob["score"]) & (ob["token"] != 2)
+        lse_o = orc.step(x_np)
+        out = stepper.step(x_dev, row_lse_in=torch.from_numpy(lse_o).cuda())
+        g = gpu_beam(out)
+        assert_beam_equal(g, orc.beam(), f"{wl.name} step {t}")
+        err = np.abs(g["row_lse"][open_rows].astype(np.float64) - lse_o[open_rows]).max() if open_rows.any() else 0.0
+        worst = max(worst, float(err))
+        assert err <= lse_tol, f"{wl.name} step {t}: row normaliser off by {err}"
+        assert (g["row_lse"][~open_rows] == 0).all()
+    return orc, worst
+
+
+def assert_finalize_equal(stepper, orc):
+    tokens, length, score, flags = stepper.finalize()
+    for b, (toks, sc, done) in enumerate(orc.finalize()):
+        assert length[b] == len(toks) and tokens[b, :length[b]].tolist() == toks, f"sentence {b}: tokens differ"
+        assert (tokens[b, length[b]:] == 0).all()
+        assert bool(flags[b] & 1) == done and (score[b] == np.float32(sc) or (np.isinf(score[b]) and np.isinf(sc)))

@@ -414,3 +414,18 @@ def test_length_normalisation_divides_completed_scores_by_their_length():
     fin = [h for h in range(3) if np.isfinite(bm["score"][h]) and bm["token"][h] == 2]
     assert done and any(bm["len"][h] == len(toks) and np.float32(bm["score"][h] / np.float32(len(toks))) == score
                         for h in fin)
+
+
+def test_row_top_is_a_stable_descending_sort():
+    rng = np.random.default_rng(17)
+    for V, n in [(1, 3), (5, 5), (40, 7), (300, 22)]:
+        for quant in (False, True):
+            x = rng.normal(0, 2, V).astype(np.float32)
+            if quant:
+                x = np.round(x)
+                x[rng.integers(0, V)] = NEG
+            val, idx = O.row_top(x, n)
+            order = np.argsort(-x, kind="stable")[:n]
+            m = min(n, V)
+            assert idx[:m].tolist() == order.tolist() and np.array_equal(val[:m], x[order])
+            assert (idx[m:] == -1).all() and np.isinf(val[m:]).all()
