@@ -85,3 +85,61 @@ def assert_finalize_equal(stepper, orc):
         assert length[b] == len(toks) and tokens[b, :length[b]].tolist() == toks, f"sentence {b}: tokens differ"
         assert (tokens[b, length[b]:] == 0).all()
         assert bool(flags[b] & 1) == done and (score[b] == np.float32(sc) or (np.isinf(score[b]) and np.isinf(sc)))
+
+
+def check_beam_invariants(g, wl, C_per_sentence, where):
+    """Properties every beam must have whatever the tie-breaks were (Sections 3.1-3.3)."""
+    k = wl.k
+    for b in range(wl.B):
+        s = slice(b * k, (b + 1) * k)
+        sc = g["score"][s]
+        live = np.isfinite(sc)
+        assert (np.diff(live.astype(int)) <= 0).all(), f"{where}: empty slot before a live one (sentence {b})"
+        assert (np.diff(sc[live]) <= 0).all(), f"{where}: beam not in decreasing order (sentence {b})"
+        pc = np.array([bin(int(m)).count("1") for m in g["met_mask"][s]])
+        assert (g["bank"][s][live] == pc[live]).all() and (g["bank"][s][~live] == -1).all()
+        fin = live & (g["token"][s] == 2)
+        assert (pc[fin] == C_per_sentence[b]).all(), f"{where}: end token before all constraints (sentence {b})"
+        assert ((g["backptr"][s] >= 0) & (g["backptr"][s] < k)).all()
+
+
+def free_run(wl, stepper, sample, steps, gpu_gen, threads=8, score_tol=1e-5):
+    """The CUDA library in its own closed loop over the whole workload (its own normalisers, logits generated
+    from its own beam), next to independent oracle runs of the sampled sentences.  Sentences must match
+    exactly; where a sampled sentence first differs, the two beams must hold the same scores rank by rank
+    within the accumulated tolerance (a tie decided by the last bit of a normaliser), and the sentence leaves
+    the comparison.  Returns (compared sentence-steps, sentences that left)."""
+    import torch
+    sub = wl.subset(sample)
+    orc = O.Batch(sub.k, sub.V, steps, sub.constraints, threads=threads)
+    host_gen = LogitStream(sub)
+    C_all = [sum(len(p) for p in c) for c in wl.constraints]
+    k = wl.k
+    tok = torch.full((wl.R,), 0, dtype=torch.int32, device="cuda"); tok[::k] = 1
+    mask = torch.zeros(wl.R, dtype=torch.int64, device="cuda")
+    alive = [True] * len(sample)
+    compared = 0
+    for t in range(steps):
+        x_dev = gpu_gen.step_logits(t, tok, mask)
+        out = stepper.step(x_dev)
+        tok, mask = out["token"].clone(), out["met_mask"].clone()
+        g = gpu_beam(out)
+        check_beam_invariants(g, wl, C_all, f"{wl.name} step {t}")
+        ob = orc.beam()
+        orc.step(host_gen.step_logits(t, ob["token"], ob["met_mask"]))
+        ob = orc.beam()
+        for i, b in enumerate(sample):
+            if not alive[i]:
+                continue
+            gs = {f: g[f][b * k:(b + 1) * k] for f in BEAM_FIELDS + ("score",)}
+            os_ = {f: ob[f][i * k:(i + 1) * k] for f in BEAM_FIELDS + ("score",)}
+            tol = score_tol * (t + 1)
+            fin = np.isfinite(os_["score"])
+            assert (np.isfinite(gs["score"]) == fin).all(), f"step {t} sentence {b}: live slots differ"
+            assert np.abs(gs["score"][fin] - os_["score"][fin]).max(initial=0) <= tol, \
+                f"step {t} sentence {b}: scores differ beyond {tol}"
+            if all((gs[f] == os_[f]).all() for f in BEAM_FIELDS):
+                compared += 1
+            else:
+                alive[i] = False
+    return compared, alive.count(False)

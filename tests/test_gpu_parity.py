@@ -109,3 +109,167 @@ def test_step_parity_phrasal(dba):
     st = _stepper(dba, wl)
     orc, worst = lockstep(wl, st)
     assert_finalize_equal(st, orc)
+
+
+def test_step_parity_ragged(dba):
+    from synth_inputs.gpu import GpuLogitStream
+    wl = make_workload("ragged")
+    st = _stepper(dba, wl)
+    orc, worst = lockstep(wl, st, gpu_gen=GpuLogitStream(wl))
+    assert_finalize_equal(st, orc)
+
+
+@pytest.mark.parametrize("C", [1, 5, 10, 20, 50])
+def test_step_parity_scaling(dba, C):
+    from synth_inputs.gpu import GpuLogitStream
+    wl = make_workload("scaling", C=C)
+    st = _stepper(dba, wl, steps=40)
+    orc, worst = lockstep(wl, st, steps=40, gpu_gen=GpuLogitStream(wl))
+    assert_finalize_equal(st, orc)
+
+
+def test_step_parity_serving_sampled_sentences(dba):
+    """Eight of the 256 sentences of the serving workload, all 120 steps, as a batch of their own."""
+    from synth_inputs.gpu import GpuLogitStream
+    wl = make_workload("serving").subset([0, 31, 64, 100, 129, 177, 200, 255])
+    st = _stepper(dba, wl)
+    orc, worst = lockstep(wl, st, gpu_gen=GpuLogitStream(wl))
+    assert_finalize_equal(st, orc)
+    assert sum(done for _, _, done in orc.finalize()) >= 6        # the stream lets most sentences finish
+
+
+def test_serving_full_size_free_run_against_sampled_oracle(dba):
+    """The launch configuration the benchmark times (B=256, k=20, V=64000, bf16), free-running."""
+    from synth_inputs.gpu import GpuLogitStream
+    from tests.parity import free_run
+    wl = make_workload("serving")
+    st = _stepper(dba, wl)
+    steps = 30
+    compared, left = free_run(wl, st, [3, 77, 140, 201, 254], steps, GpuLogitStream(wl))
+    assert left <= 1 and compared >= 4 * steps
+
+
+# ------------------------------------------------------------------------------------------ edge cases
+def _custom(name, B, k, V, steps, constraints, dtype="f32", zipf=True):
+    from synth_inputs.configs import Workload
+    return Workload(name=name, cfg_id=9, B=B, k=k, V=V, steps=steps, dtype=dtype, zipf=zipf, boost=True,
+                    constraints=constraints, seed=0, sent_ids=np.arange(B, dtype=np.int64))
+
+
+EDGE = {
+    "beam_of_one":            dict(B=2, k=1, V=300, steps=12, constraints=[[[5], [6, 7]], []]),
+    "no_constraints":         dict(B=3, k=4, V=517, steps=10, constraints=[[], [], []]),
+    "more_constraints_than_beam": dict(B=2, k=3, V=400, steps=16, constraints=[[[w] for w in range(10, 20)], [[30, 31, 32, 33], [40], [41]]]),
+    "sixty_four_constraints": dict(B=1, k=4, V=700, steps=20, constraints=[[[w] for w in range(100, 164)]]),
+    "sixty_four_in_phrases":  dict(B=1, k=6, V=700, steps=20, constraints=[[list(range(100 + 4 * i, 104 + 4 * i)) for i in range(16)]]),
+    "odd_vocab_f32":          dict(B=2, k=5, V=1003, steps=10, constraints=[[[5, 6]], [[7]]]),
+    "odd_vocab_bf16":         dict(B=2, k=5, V=1001, steps=10, constraints=[[[5, 6]], [[7]]], dtype="bf16"),
+    "duplicate_tokens":       dict(B=1, k=5, V=200, steps=12, constraints=[[[9], [9], [9, 10], [10, 9, 11]]]),
+    "self_overlapping_phrase": dict(B=1, k=6, V=120, steps=14, constraints=[[[8, 8, 9], [8, 9]]]),
+    "big_beam":               dict(B=2, k=64, V=2048, steps=8, constraints=[[[5, 6], [7]], [[9]]], dtype="bf16"),
+    "plain_normal_rows":      dict(B=2, k=7, V=900, steps=10, constraints=[[[5]], [[6, 7, 8]]], zipf=False),
+}
+
+
+@pytest.mark.parametrize("case", sorted(EDGE))
+def test_step_parity_edge_cases(dba, case):
+    p = dict(EDGE[case])
+    wl = _custom(case, **p)
+    st = _stepper(dba, wl)
+    orc, worst = lockstep(wl, st)
+    assert_finalize_equal(st, orc)
+
+
+@pytest.mark.parametrize("flags", [1, 2, 3])
+def test_flags_adjust_off_and_length_norm(dba, flags):
+    wl = make_workload("ragged", B=6, V=3000, steps=50)
+    st = _stepper(dba, wl, flags=flags)
+    orc, worst = lockstep(wl, st, flags=flags)
+    assert_finalize_equal(st, orc)
+
+
+def test_rows_with_minus_inf_and_quantised_logits(dba):
+    """Heavy ties (a few distinct values per row) and -inf holes, for both dtypes."""
+    rng = np.random.default_rng(5)
+    for dtype in ("f32", "bf16"):
+        wl = _custom("holes", 3, 5, 260, 9, [[[5, 6], [7]], [[8]], []], dtype=dtype)
+        st = _stepper(dba, wl)
+        orc = O.Batch(wl.k, wl.V, wl.steps, wl.constraints)
+        for t in range(wl.steps):
+            x = np.round(rng.normal(0, 1.5, (wl.R, wl.V))).astype(np.float32) + np.float32(0.0)
+            x[rng.random(x.shape) < 0.4] = -np.inf
+            x[:, 2] = -30.0 if t < 5 else 3.0
+            if dtype == "bf16":
+                x_np = (x.view(np.uint32) >> 16).astype(np.uint16)       # small integers are exact in bf16
+            else:
+                x_np = x
+            lse_o = orc.step(x_np)
+            out = st.step(to_device_logits(x_np, wl), row_lse_in=torch.from_numpy(lse_o).cuda())
+            assert_beam_equal(gpu_beam(out), orc.beam(), f"holes {dtype} step {t}")
+        assert_finalize_equal(st, orc)
+
+
+def test_scores_that_round_together_across_the_row_cut(dba):
+    """Logits one ulp apart collapse onto a few fp32 scores; the cells kept must then be the lowest token ids
+    among the equal scores, also beyond the k+2 entries the row scan keeps."""
+    k, V = 4, 96
+    wl = _custom("collapse", 1, k, V, 3, [[]])
+    st = _stepper(dba, wl)
+    orc = O.Batch(k, V, 3, wl.constraints)
+    for t in range(3):
+        base = np.float32(1.0)
+        ulps = np.arange(V, dtype=np.int32)[::-1].copy()             # higher logits at lower... reversed below
+        x = (base.view(np.int32) + ulps).view(np.float32)           # descending by index, 1 ulp steps
+        x = x[::-1].copy()                                           # ascending: best raw logits have the HIGHEST ids
+        x = np.tile(x, (k, 1)).astype(np.float32)
+        x[:, 2] = -50.0
+        lse_o = orc.step(x)
+        out = st.step(torch.from_numpy(x).cuda(), row_lse_in=torch.from_numpy(lse_o).cuda())
+        assert_beam_equal(gpu_beam(out), orc.beam(), f"collapse step {t}")
+    sc = orc.beam()["score"]
+    assert len(np.unique(sc)) < k                                   # the case really had equal scores
+
+
+def test_step_host_equals_step_and_reset_replays(dba):
+    wl = make_workload("ragged", B=4, V=2000, steps=12)
+    gen = LogitStream(wl)
+    a = _stepper(dba, wl)
+    b = _stepper(dba, wl, flags=dba.FLAG_HOST_STAGING)
+    host_out = b.new_outputs(host=True)
+    tok = np.zeros(wl.R, np.int32); tok[::wl.k] = 1
+    mask = np.zeros(wl.R, np.uint64)
+    trace = []
+    for t in range(wl.steps):
+        x = gen.step_logits(t, tok, mask)
+        ga = gpu_beam(a.step(to_device_logits(x, wl)))
+        xh = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory()
+        b.step_host(xh, host_out)
+        gb = {f: host_out[f].numpy().copy() for f in host_out}
+        gb["met_mask"] = gb["met_mask"].view(np.uint64)
+        assert_beam_equal(gb, ga, f"host step {t}", fields=("backptr", "token", "bank", "met_mask", "active", "score", "row_lse"))
+        trace.append((x, ga))
+        tok, mask = ga["token"], ga["met_mask"]
+    fa = a.finalize()
+    a.reset()
+    for t, (x, want) in enumerate(trace):
+        assert_beam_equal(gpu_beam(a.step(to_device_logits(x, wl))), want, f"replay step {t}",
+                          fields=("backptr", "token", "bank", "met_mask", "active", "score", "row_lse"))
+    for u, v in zip(fa, a.finalize()):
+        assert np.array_equal(u, v)
+    with pytest.raises(dba.DbaError) as e:
+        a.step(to_device_logits(trace[0][0], wl))
+    assert e.value.code == 3                                        # DBA_ERR_STATE: past max_steps
+
+
+def test_argument_errors_are_reported_not_launched(dba):
+    mk = lambda **kw: dba.DbaStepper(**{**dict(B=1, k=2, V=50, max_steps=3, constraints=[[[5]]]), **kw})
+    for kw, code in [(dict(k=65), 2), (dict(constraints=[[[w] for w in range(4, 69)]], V=100), 2),
+                     (dict(constraints=[[[2]]]), 1), (dict(constraints=[[[50]]]), 1), (dict(constraints=[[[]]]), 1),
+                     (dict(k=0), 1), (dict(V=2**31 // 2, k=2), 2), (dict(dtype=7), 1), (dict(eos=99), 1)]:
+        with pytest.raises(dba.DbaError) as e:
+            mk(**kw)
+        assert e.value.code == code, kw
+    st = mk()
+    with pytest.raises(dba.DbaError) as e:
+        st.step_host(torch.zeros(2, 50), st.new_outputs(host=True))
+    assert e.value.code == 3                                        # no staging area was requested
