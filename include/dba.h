@@ -147,6 +147,16 @@ dba_status dba_step_host(dba_handle* h, const void* logits_host, int64_t row_str
 dba_status dba_finalize(dba_handle* h, int32_t* tokens_host, int32_t* len_host, float* score_host,
                         int32_t* flags_host);
 
+/*
+ * Optional per-kernel timing for benchmarks.  While enabled, dba_step brackets each of its three kernels
+ * (row scan; candidates; allocation) with CUDA events on the handle's stream.  dba_timing_read waits for
+ * the stream, adds up the elapsed milliseconds of every step recorded since the last read into
+ * ms_total[0..2], stores the number of steps in *steps and clears the record.  At most 4096 steps are
+ * kept between reads (further steps are not recorded).  Off by default.
+ */
+dba_status dba_timing_enable(dba_handle* h, int32_t on);
+dba_status dba_timing_read(dba_handle* h, double ms_total[3], int64_t* steps);
+
 /* Number of kernels this handle has launched so far (for accounting in benchmarks). */
 uint64_t dba_launch_count(const dba_handle* h);
 

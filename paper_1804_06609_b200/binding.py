@@ -15,7 +15,7 @@ F32, BF16 = 0, 1
 FLAG_ADJUST_OFF, FLAG_LENGTH_NORM, FLAG_HOST_STAGING = 1, 2, 4
 
 EXPORTS = ["dba_workspace_bytes", "dba_init", "dba_reset", "dba_step", "dba_step_host", "dba_finalize",
-           "dba_launch_count", "dba_destroy", "dba_status_string", "dba_row_scan_scratch_bytes", "dba_row_scan"]
+           "dba_timing_enable", "dba_timing_read", "dba_launch_count", "dba_destroy", "dba_status_string", "dba_row_scan_scratch_bytes", "dba_row_scan"]
 
 
 class DbaError(RuntimeError):
@@ -53,6 +53,8 @@ def lib():
         L.dba_step.argtypes = [vp, vp, C.c_int64, vp, C.POINTER(StepOut)]
         L.dba_step_host.argtypes = [vp, vp, C.c_int64, C.POINTER(StepOut)]
         L.dba_finalize.argtypes = [vp, vp, vp, vp, vp]
+        L.dba_timing_enable.argtypes = [vp, C.c_int32]
+        L.dba_timing_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.dba_launch_count.argtypes = [vp]
         L.dba_launch_count.restype = C.c_uint64
         L.dba_destroy.argtypes = [vp]
@@ -159,6 +161,15 @@ class DbaStepper:
         _check(lib().dba_finalize(self._h, tokens.ctypes.data, length.ctypes.data, score.ctypes.data, flags.ctypes.data),
                "dba_finalize")
         return tokens, length, score, flags
+
+    def timing_enable(self, on=True):
+        _check(lib().dba_timing_enable(self._h, int(on)), "dba_timing_enable")
+
+    def timing_read(self):
+        """(ms of [row scan, candidates, allocation] summed over the recorded steps, number of steps)."""
+        ms = (C.c_double * 3)(); n = C.c_int64()
+        _check(lib().dba_timing_read(self._h, ms, C.byref(n)), "dba_timing_read")
+        return list(ms), n.value
 
     def launch_count(self):
         return int(lib().dba_launch_count(self._h))

@@ -33,7 +33,13 @@ struct dba_handle {
     int cur;
     int launches_tmp;
     uint64_t launches;
+    // optional kernel timing
+    bool timing;
+    std::vector<cudaEvent_t> ev;   // 4 events per recorded step
+    int ev_steps;
 };
+
+constexpr int kTimingCap = 4096;
 
 namespace {
 
@@ -222,15 +228,33 @@ dba_status dba_step(dba_handle* h, const void* logits_dev, int64_t row_stride_el
     const Beam& cur = h->beam[h->cur];
     const Beam& nxt = h->beam[h->cur ^ 1];
     h->launches_tmp = 0;
-    cudaError_t e = launch_row_scan(logits_dev, row_stride_elems, h->d, cur.score, cur.token, h->part, h->status,
-                                    h->stream, &h->launches_tmp);
+    cudaEvent_t* ev = nullptr;
+    if (h->timing && h->ev_steps < kTimingCap) {
+        if ((int)h->ev.size() < 4 * (h->ev_steps + 1)) {
+            for (int i = 0; i < 4; ++i) {
+                cudaEvent_t x;
+                if (cudaEventCreate(&x) != cudaSuccess) return DBA_ERR_CUDA;
+                h->ev.push_back(x);
+            }
+        }
+        ev = &h->ev[4 * h->ev_steps];
+        h->ev_steps += 1;
+    }
+    cudaError_t e = cudaSuccess;
+    if (ev) e = cudaEventRecord(ev[0], h->stream);
+    if (e == cudaSuccess)
+        e = launch_row_scan(logits_dev, row_stride_elems, h->d, cur.score, cur.token, h->part, h->status,
+                            h->stream, &h->launches_tmp);
+    if (ev && e == cudaSuccess) e = cudaEventRecord(ev[1], h->stream);
     if (e == cudaSuccess)
         e = launch_candidates(logits_dev, row_stride_elems, h->d, h->cons, cur, h->part, row_lse_in_dev, h->row_lse,
                               h->cand, h->ncand, h->bank_count, h->status, h->stream, &h->launches_tmp);
+    if (ev && e == cudaSuccess) e = cudaEventRecord(ev[2], h->stream);
     if (e == cudaSuccess)
         e = launch_allocate(h->d, h->cons, cur, nxt, h->cand, h->ncand, h->bank_count, h->row_lse, out,
                             h->hist_bp + (size_t)h->t * h->d.R, h->hist_tok + (size_t)h->t * h->d.R, h->stream,
                             &h->launches_tmp);
+    if (ev && e == cudaSuccess) e = cudaEventRecord(ev[3], h->stream);
     h->launches += h->launches_tmp;
     if (e != cudaSuccess) return DBA_ERR_CUDA;
     h->cur ^= 1;
@@ -293,9 +317,34 @@ dba_status dba_finalize(dba_handle* h, int32_t* tokens_host, int32_t* len_host, 
     return DBA_OK;
 }
 
+dba_status dba_timing_enable(dba_handle* h, int32_t on) {
+    if (!h) return DBA_ERR_INVALID_ARG;
+    h->timing = on != 0;
+    return DBA_OK;
+}
+
+dba_status dba_timing_read(dba_handle* h, double ms_total[3], int64_t* steps) {
+    if (!h || !ms_total || !steps) return DBA_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) return DBA_ERR_CUDA;
+    ms_total[0] = ms_total[1] = ms_total[2] = 0.0;
+    for (int i = 0; i < h->ev_steps; ++i)
+        for (int j = 0; j < 3; ++j) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, h->ev[4 * i + j], h->ev[4 * i + j + 1]) != cudaSuccess) return DBA_ERR_CUDA;
+            ms_total[j] += ms;
+        }
+    *steps = h->ev_steps;
+    h->ev_steps = 0;
+    return DBA_OK;
+}
+
 uint64_t dba_launch_count(const dba_handle* h) { return h ? h->launches : 0; }
 
-void dba_destroy(dba_handle* h) { delete h; }
+void dba_destroy(dba_handle* h) {
+    if (!h) return;
+    for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
+    delete h;
+}
 
 const char* dba_status_string(dba_status s) {
     switch (s) {
