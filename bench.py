@@ -1,0 +1,309 @@
+#!/usr/bin/env python
+"""Benchmark of the DBA step on the serving-scale workload (B=256, k=20, V=64000, bf16, 120-step stream).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A step is one dba_step call: all three kernels over one batch of logits.  The logit stream is generated
+once, untimed, by running the step in closed loop (every row depends on the hypothesis' last token), and
+kept resident in HBM; the timed loop then replays it, resetting the beam whenever the stream wraps.
+One JSON line is printed by rank 0.  With N > 1 every rank runs an independent replica (sentences do not
+interact, the path has no collective); the value is the sum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "dba_steps_per_sec"
+L2_BYTES = 126 * 2**20
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1200)
+    ap.add_argument("--warmup", type=int, default=120)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="serving")
+    ap.add_argument("--C", type=int, default=None, help="constraint count of the 'scaling' workload")
+    ap.add_argument("--e2e-steps", type=int, default=16)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def ncu_traffic(workload):
+    """DRAM bytes per row-scan launch from the last ncu capture, if the kernel has not changed since."""
+    p = os.path.join(ROOT, "profiles", "row_scan_traffic.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return d.get(workload)
+    return None
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.stop_flag, self.sm, self.reasons, self.max_mhz = index, False, [], set(), None
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                     nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                     nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                     nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
+            while not self.stop_flag:
+                self.sm.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+                time.sleep(0.01)
+        except Exception as e:  # NVML missing: report that no clocks were seen
+            self.reasons.add(f"nvml_unavailable:{type(e).__name__}")
+
+    def result(self):
+        import statistics
+        return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+def workload_of(args):
+    from synth_inputs import make_workload
+    return make_workload(args.workload, C=args.C)
+
+
+# ---------------------------------------------------------------------------------------------- oracle
+def oracle_rate(wl, n_sent, steps, warmup=0, budget_s=None):
+    """Times the CPU oracle, as it stands, single-threaded, on the first n_sent sentences of the workload in
+    closed loop.  Returns (whole-batch steps/s equivalent, seconds timed, steps timed)."""
+    from oracle import dba_oracle as O
+    from synth_inputs import LogitStream
+    sub = wl.subset(range(n_sent))
+    gen = LogitStream(sub)
+    orc = O.Batch(sub.k, sub.V, wl.steps, sub.constraints, threads=1)
+    t_spent, done, t_in = 0.0, 0, 0
+    for i in range(warmup + steps):
+        if t_in == wl.steps:
+            orc = O.Batch(sub.k, sub.V, wl.steps, sub.constraints, threads=1); t_in = 0
+        b = orc.beam()
+        x = gen.step_logits(t_in, b["token"], b["met_mask"])       # input generation is not timed
+        t0 = time.perf_counter()
+        orc.step(x)
+        dt = time.perf_counter() - t0
+        t_in += 1
+        if i >= warmup:
+            t_spent += dt; done += 1
+            if budget_s is not None and t_spent > budget_s:
+                break
+    per_sentence_step = t_spent / (done * n_sent)
+    return 1.0 / (per_sentence_step * wl.B), t_spent, done
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = workload_of(args)
+    total = args.steps + args.warmup
+    per_sentence = 0.003 * wl.k * wl.V / 64000 * (wl.k / 20) + 0.002     # rough seconds per sentence-step
+    n_sent = max(1, min(wl.B, 16, int(150.0 / (total * per_sentence))))
+    value, secs, done = oracle_rate(wl, n_sent, args.steps, args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": value,
+            "unit": f"steps/s (one step = {wl.R} hypotheses x {wl.V} logits)", "n_gpus": args.gpus,
+            "steps": done, "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "k": wl.k, "V": wl.V, "logits": wl.dtype},
+            "cpu_baseline": {"value": value, "unit": "steps/s", "cores": 1, "kind": "oracle",
+                             "sample": f"{n_sent} of {wl.B} sentences per step, {done} steps of the stream, "
+                                       f"scaled by {wl.B}/{n_sent}"},
+            "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------- ours
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_1804_06609_b200 as pkg
+    from synth_inputs.gpu import GpuLogitStream
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    pkg.lib()
+
+    wl = workload_of(args)
+    if world > 1:                                   # replicas: every rank gets its own sentences
+        import numpy as np
+        wl.sent_ids = wl.sent_ids + np.int64(rank * wl.B)
+    esize = 2 if wl.dtype == "bf16" else 4
+    step_bytes = wl.R * wl.V * esize
+    free, _ = torch.cuda.mem_get_info(dev)
+    T = int(max(1, min(wl.steps, (free * 0.6) // step_bytes)))
+    # rotate enough distinct step buffers that consecutive steps never find their input in L2
+    gen = GpuLogitStream(wl, dev)
+    st = pkg.DbaStepper(wl.B, wl.k, wl.V, wl.steps, constraints=wl.constraints,
+                        dtype=pkg.BF16 if wl.dtype == "bf16" else pkg.F32, device=dev)
+    logits = torch.empty(T, wl.R, wl.V, dtype=gen.tdtype, device=dev)
+
+    # --- untimed: generate the stream in closed loop, count the rows that are open at each step -------
+    tok = torch.zeros(wl.R, dtype=torch.int32, device=dev); tok[::wl.k] = 1
+    mask = torch.zeros(wl.R, dtype=torch.int64, device=dev)
+    open_rows = []
+    for t in range(T):
+        open_rows.append(wl.B if t == 0 else int(((out["score"] > float("-inf")) & (out["token"] != 2)).sum()))
+        gen.step_logits(t, tok, mask, out=logits[t])
+        out = st.step(logits[t])
+        tok, mask = out["token"], out["met_mask"]
+    tokens, length, score, flags = st.finalize()
+    completed = int((flags & 1).sum())
+
+    def replay(n, start=0):
+        for i in range(start, start + n):
+            t = i % T
+            if t == 0:
+                st.reset()
+            st.step(logits[t])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    # --- timed: K steps, device clock, max over ranks ---------------------------------------------------
+    replay(args.warmup)
+    launches0 = st.launch_count()
+    sampler = ClockSampler(local); sampler.start()
+    time.sleep(0.05)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    replay(args.steps, start=args.warmup)
+    e1.record()
+    barrier()
+    sampler.stop_flag = True; sampler.join()
+    ms = e0.elapsed_time(e1)
+    launches = st.launch_count() - launches0
+    if world > 1:
+        tms = torch.tensor([ms], device=dev); dist.all_reduce(tms, op=dist.ReduceOp.MAX); ms = float(tms)
+    value = world * args.steps / (ms / 1e3)
+
+    # --- per-kernel time of the same replay (events inside the library, on its stream) -----------------
+    st.timing_enable(True)
+    kt, ksteps, kbytes = [0.0, 0.0, 0.0], 0, 0
+    pos = args.warmup + args.steps
+    remaining = args.steps
+    while remaining > 0:
+        n = min(remaining, 2048)
+        replay(n, start=pos)
+        part, cnt = st.timing_read()
+        kt = [a + b for a, b in zip(kt, part)]; ksteps += cnt
+        kbytes += sum(open_rows[i % T] for i in range(pos, pos + n)) * wl.V * esize
+        pos += n; remaining -= n
+    st.timing_enable(False)
+    peak, peak_kind = measured_peak()
+    scan_ms = kt[0] / ksteps
+    achieved = kbytes / ksteps / (scan_ms / 1e3) / 1e9
+    traffic = ncu_traffic(wl.name)
+
+    # --- end to end: host logits in pinned memory, outputs read back, through dba_step_host ------------
+    Th = min(T, 8)
+    ste = pkg.DbaStepper(wl.B, wl.k, wl.V, wl.steps, constraints=wl.constraints,
+                         dtype=pkg.BF16 if wl.dtype == "bf16" else pkg.F32, device=dev,
+                         flags=pkg.FLAG_HOST_STAGING)
+    host = torch.empty(Th, wl.R, wl.V, dtype=gen.tdtype, pin_memory=True)
+    host.copy_(logits[:Th])
+    host_out = ste.new_outputs(host=True)
+    d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+
+    def replay_host(n):
+        for i in range(n):
+            if i % Th == 0:
+                ste.reset()
+            ste.step_host(host[i % Th], host_out)
+
+    replay_host(3)
+    barrier()
+    t0 = time.perf_counter()
+    replay_host(args.e2e_steps)
+    torch.cuda.synchronize(dev)
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        te = torch.tensor([e2e_s], device=dev); dist.all_reduce(te, op=dist.ReduceOp.MAX); e2e_s = float(te)
+    e2e_value = world * args.e2e_steps / e2e_s
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        n_sent = 8
+        v, secs, done = oracle_rate(wl, n_sent, 24, warmup=0, budget_s=20.0)
+        cpu = {"value": v, "unit": "steps/s", "cores": 1, "kind": "oracle",
+               "sample": f"first {n_sent} of {wl.B} sentences, steps 0-{done - 1} of the stream in closed loop, "
+                         f"{secs:.1f} s of oracle time, scaled by {wl.B}/{n_sent}"}
+    unit = f"steps/s (one step = {wl.R} hypotheses x {wl.V} {wl.dtype} logits per GPU)"
+    line = {
+        "metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "B": wl.B, "k": wl.k, "V": wl.V, "logits": wl.dtype,
+                   "constraint_tokens_per_sentence": sorted({sum(len(p) for p in c) for c in wl.constraints}),
+                   "stream_steps": T, "open_rows_mean": sum(open_rows) / T, "rows": wl.R,
+                   "completed_sentences": completed,
+                   "l2": f"inputs larger than L2: {step_bytes >> 20} MiB of logits per step, {T} step buffers"
+                         if step_bytes > L2_BYTES else f"{T} rotating step buffers, {T * step_bytes >> 20} MiB in all",
+                   "parallelism": "replicas" if world > 1 else "single GPU"},
+        "hyp_steps_per_sec": value * wl.R,
+        "kernel_ms": {"row_scan": scan_ms, "candidates": kt[1] / ksteps, "allocate": kt[2] / ksteps},
+        "roofline": {"bound": "hbm", "kernel": "row_scan", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs_nominal": achieved / 8000.0,
+                     "algorithmic_bytes_per_launch": kbytes / ksteps, "traffic": traffic},
+        "e2e": {"value": e2e_value, "unit": "steps/s", "h2d_bytes_per_step": step_bytes, "d2h_bytes_per_step": d2h,
+                "steps": args.e2e_steps},
+        "gpu_launches": launches,
+        "clocks": sampler.result(),
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
