@@ -178,6 +178,28 @@ dba_status dba_row_scan(const void* logits_dev, int32_t logit_dtype, int32_t R, 
                         int64_t row_stride_elems, int32_t n_top, void* scratch_dev, size_t scratch_bytes,
                         float* row_lse_dev, float* top_val_dev, int32_t* top_idx_dev, void* cuda_stream);
 
+/*
+ * dba_row_scan for callers that cannot allocate device memory (the paper has no counterpart: this is a
+ * packaging variant of the entry point above, not a step of the method).  Use it where cudaMalloc is not
+ * an option: a serving process whose memory pool is fixed at start-up, a plug-in that receives buffers but
+ * owns no allocator, a latency path that must not risk the device-wide synchronisation an allocation can
+ * cause.  The scratch that dba_row_scan takes from the caller lives here in a fixed array inside the
+ * library image: 4 MiB (dba_row_scan_static_max_bytes) on every GPU that loads the library, for as long as
+ * the process runs.  Inputs, outputs and results are those of dba_row_scan.
+ *   - A problem whose scratch need (dba_row_scan_scratch_bytes) exceeds the fixed size is refused with
+ *     DBA_ERR_UNSUPPORTED and nothing is launched.
+ *   - No device memory is allocated or freed, here or in anything this function calls.
+ *   - The first call on each device looks up the array's device address (with that device current); make
+ *     that first call outside any stream capture.
+ *   - All calls on one device share the one array.  Each call overwrites what it later reads, so calls
+ *     that follow one another on a stream are independent; calls that can overlap on the GPU (different
+ *     streams, no ordering between them) race on it and give undefined results.
+ */
+dba_status dba_row_scan_static(const void* logits_dev, int32_t logit_dtype, int32_t R, int32_t V,
+                               int64_t row_stride_elems, int32_t n_top, float* row_lse_dev,
+                               float* top_val_dev, int32_t* top_idx_dev, void* cuda_stream);
+size_t dba_row_scan_static_max_bytes(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -15,7 +15,8 @@ F32, BF16 = 0, 1
 FLAG_ADJUST_OFF, FLAG_LENGTH_NORM, FLAG_HOST_STAGING = 1, 2, 4
 
 EXPORTS = ["dba_workspace_bytes", "dba_init", "dba_reset", "dba_step", "dba_step_host", "dba_finalize",
-           "dba_timing_enable", "dba_timing_read", "dba_launch_count", "dba_destroy", "dba_status_string", "dba_row_scan_scratch_bytes", "dba_row_scan"]
+           "dba_timing_enable", "dba_timing_read", "dba_launch_count", "dba_destroy", "dba_status_string", "dba_row_scan_scratch_bytes", "dba_row_scan",
+           "dba_row_scan_static", "dba_row_scan_static_max_bytes"]
 
 
 class DbaError(RuntimeError):
@@ -64,6 +65,8 @@ def lib():
         L.dba_row_scan_scratch_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_size_t)]
         L.dba_row_scan.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int32, vp, C.c_size_t,
                                    vp, vp, vp, vp]
+        L.dba_row_scan_static.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int32, vp, vp, vp, vp]
+        L.dba_row_scan_static_max_bytes.restype = C.c_size_t
         _lib = L
     return _lib
 
@@ -201,3 +204,14 @@ def row_scan(logits, n_top, stream=None):
                               val.data_ptr(), idx.data_ptr(), st.cuda_stream), "dba_row_scan")
     st.synchronize()          # the scratch tensor must outlive the kernels
     return lse, val, idx
+
+
+def row_scan_static(logits, n_top, lse, val, idx, stream=None):
+    """dba_row_scan_static: like row_scan, but the library's built-in scratch is used and the caller brings the
+    output tensors (lse [R] f32, val [R, n_top] f32, idx [R, n_top] i32).  Nothing is allocated here."""
+    import torch
+    R, V = logits.shape
+    st = stream if stream is not None else torch.cuda.current_stream(logits.device)
+    _check(lib().dba_row_scan_static(logits.data_ptr(), _dtype_code(logits), R, V, logits.stride(0), n_top,
+                                     lse.data_ptr(), val.data_ptr(), idx.data_ptr(), st.cuda_stream),
+           "dba_row_scan_static")
