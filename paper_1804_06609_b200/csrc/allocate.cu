@@ -27,7 +27,7 @@ __global__ void __launch_bounds__(kAllocWarps * 32)
 allocate_kernel(Dims d, const SentCons* __restrict__ cons, Beam cur, Beam nxt, const Cand* __restrict__ cand,
                 const int32_t* __restrict__ ncand, const int32_t* __restrict__ bank_count,
                 const float* __restrict__ row_lse, dba_step_out out, int32_t* __restrict__ hist_bp,
-                int32_t* __restrict__ hist_tok) {
+                int32_t* __restrict__ hist_tok, int32_t* __restrict__ open_list, int32_t* __restrict__ open_count) {
     __shared__ int s_n[kAllocWarps][kBanks];
     __shared__ int s_alloc[kAllocWarps][kBanks];
     __shared__ int s_off[kAllocWarps][kBanks];
@@ -129,16 +129,29 @@ allocate_kernel(Dims d, const SentCons* __restrict__ cons, Beam cur, Beam nxt, c
     }
     if (out.row_lse)
         for (int i = lane; i < k; i += 32) out.row_lse[r0 + i] = row_lse[r0 + i];
+    // rows the next step has to scan: live slots that have not generated the end token
+    __syncwarp();
+    for (int i0 = 0; i0 < k; i0 += 32) {
+        const int i = i0 + lane;
+        const bool open = i < k && nxt.score[r0 + i] != neg_inf() && nxt.token[r0 + i] != d.eos_id;
+        const unsigned bal = __ballot_sync(kFullMask, open);
+        int base = 0;
+        if (lane == 0 && bal) base = atomicAdd(open_count, __popc(bal));
+        base = __shfl_sync(kFullMask, base, 0);
+        if (open) open_list[base + __popc(bal & ((1u << lane) - 1u))] = r0 + i;
+    }
 }
 
 // Algorithm 1, DECODER-INIT: slot 0 holds the start symbol at score 0, the other slots are empty.
-__global__ void reset_kernel(Dims d, Beam beam) {
+__global__ void reset_kernel(Dims d, Beam beam, int32_t* __restrict__ open_list, int32_t* __restrict__ open_count) {
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= d.R) return;
     const bool first = (r % d.k) == 0;
     beam.score[r] = first ? 0.f : neg_inf();
     beam.token[r] = first ? d.bos_id : d.pad_id;
     beam.mask[r] = 0; beam.active[r] = -1; beam.len[r] = 0; beam.bank[r] = first ? 0 : -1; beam.backptr[r] = 0;
+    if (first) open_list[r / d.k] = r;
+    if (r == 0) *open_count = d.B;
 }
 
 // Section 3.3: the completed hypothesis with the highest score (Section 4: optionally divided by its
@@ -190,15 +203,16 @@ __global__ void finalize_kernel(Dims d, Beam beam, const int32_t* __restrict__ h
 cudaError_t launch_allocate(const Dims& d, const SentCons* cons, const Beam& cur, const Beam& next,
                             const Cand* cand, const int32_t* ncand, const int32_t* bank_count,
                             const float* row_lse, const dba_step_out& out, int32_t* hist_bp, int32_t* hist_tok,
-                            cudaStream_t st, int* launches) {
+                            int32_t* open_list, int32_t* open_count, cudaStream_t st, int* launches) {
     allocate_kernel<<<(d.B + kAllocWarps - 1) / kAllocWarps, kAllocWarps * 32, 0, st>>>(
-        d, cons, cur, next, cand, ncand, bank_count, row_lse, out, hist_bp, hist_tok);
+        d, cons, cur, next, cand, ncand, bank_count, row_lse, out, hist_bp, hist_tok, open_list, open_count);
     ++*launches;
     return cudaGetLastError();
 }
 
-cudaError_t launch_reset(const Dims& d, const Beam& beam, cudaStream_t st, int* launches) {
-    reset_kernel<<<(d.R + 255) / 256, 256, 0, st>>>(d, beam);
+cudaError_t launch_reset(const Dims& d, const Beam& beam, int32_t* open_list, int32_t* open_count,
+                         cudaStream_t st, int* launches) {
+    reset_kernel<<<(d.R + 255) / 256, 256, 0, st>>>(d, beam, open_list, open_count);
     ++*launches;
     return cudaGetLastError();
 }

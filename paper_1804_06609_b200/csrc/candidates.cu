@@ -21,7 +21,7 @@ struct SortEnt {
 
 struct Layout {   // byte offsets into dynamic shared memory
     int cons, parent, lse, mask, active, kind, eos_ok, rt_score, rt_w, rt_n, rt_ptr, s1_h, s1_i, stage, merged,
-        tmp_score, tmp_w, c_score, c_flat, c_mask, c_active, bank_cnt, sort, total;
+        tmp_score, tmp_w, tmp_x, c_score, c_flat, c_mask, c_active, bank_cnt, sort, total;
     int n_sort;
 };
 
@@ -47,8 +47,9 @@ __host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand
     o = align_up(o, 8);
     L.stage = o;     o += 8 * kCandWarps * (S > 1 ? S * K1 : 0);
     L.merged = o;    o += 8 * kCandWarps * K1;
-    L.tmp_score = o; o += 4 * kCandWarps * (k + 1);
-    L.tmp_w = o;     o += 4 * kCandWarps * (k + 1);
+    L.tmp_score = o; o += 4 * kCandWarps * K1;
+    L.tmp_w = o;     o += 4 * kCandWarps * K1;
+    L.tmp_x = o;     o += 4 * kCandWarps * K1;
     o = align_up(o, 8);
     L.c_mask = o;    o += 8 * max_cand;
     L.c_score = o;   o += 4 * max_cand;
@@ -93,7 +94,7 @@ __global__ void __launch_bounds__(kCandThreads)
 candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const SentCons* __restrict__ cons,
                   Beam cur, ScanOut part, const float* __restrict__ lse_in, float* __restrict__ row_lse,
                   Cand* __restrict__ cand_out, int32_t* __restrict__ ncand_out, int32_t* __restrict__ bank_count,
-                  uint32_t* __restrict__ status) {
+                  uint32_t* __restrict__ status, int32_t* __restrict__ open_count) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int k = d.k, V = d.V, K1 = d.K1, S = d.S;
     const Layout L = make_layout(k, K1, S, d.max_cand);
@@ -140,6 +141,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     }
     if (tid <= kMaxC) bank_cnt[tid] = 0;
     if (tid == 0) { s_ncand = 0; s_ns1 = 0; }
+    if (tid == 0 && blockIdx.x == 0) *open_count = 0;   // the allocation kernel rebuilds the list of open rows
     __syncthreads();
     const int C = sc.C;
     if (tid < k) s_eos_ok[tid] = __popcll(s_mask[tid]) >= C;   // Section 3.3: end token only once all are met
@@ -148,8 +150,9 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     // ---- phase A: per row, the k best cells in (score desc, token asc) order ------------------------------
     uint64_t* stage = reinterpret_cast<uint64_t*>(smem + L.stage) + warp * (S > 1 ? S * K1 : 0);
     uint64_t* merged = reinterpret_cast<uint64_t*>(smem + L.merged) + warp * K1;
-    float* tmp_score = reinterpret_cast<float*>(smem + L.tmp_score) + warp * (k + 1);
-    int* tmp_w = reinterpret_cast<int*>(smem + L.tmp_w) + warp * (k + 1);
+    float* tmp_score = reinterpret_cast<float*>(smem + L.tmp_score) + warp * K1;
+    int* tmp_w = reinterpret_cast<int*>(smem + L.tmp_w) + warp * K1;
+    float* tmp_x = reinterpret_cast<float*>(smem + L.tmp_x) + warp * K1;
     const unsigned lt_mask = (1u << lane) - 1u;
 
     for (int h = warp; h < k; h += kCandWarps) {
@@ -203,57 +206,78 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         }
         __syncwarp();
 
-        // scores of the entries that may be generated, in list order; keep k plus one sentinel
-        int total_valid = 0;
+        // scores of the entries that may be generated, in list order
+        int total_valid = 0, finite_entries = 0;
         for (int e0 = 0; e0 < K1; e0 += 32) {
             const int e = e0 + lane;
-            bool valid = false; float scv = neg_inf(); int w = -1;
+            bool valid = false, finite = false; float scv = neg_inf(), x = neg_inf(); int w = -1;
             if (e < K1) {
                 const uint64_t key = merged[e];
                 if (key) {
-                    const float x = row_key_val(key);
+                    x = row_key_val(key);
                     w = row_key_idx(key);
-                    valid = x != neg_inf() && !(w == d.eos_id && !eos_ok) && lse != neg_inf();
+                    finite = x != neg_inf();
+                    valid = finite && !(w == d.eos_id && !eos_ok) && lse != neg_inf();
                     if (valid) scv = cell_score(x, lse, parent);
                 }
             }
             const unsigned bal = __ballot_sync(kFullMask, valid);
             const int pos = total_valid + __popc(bal & lt_mask);
-            if (valid && pos <= k) { tmp_score[pos] = scv; tmp_w[pos] = w; }
+            if (valid) { tmp_score[pos] = scv; tmp_w[pos] = w; tmp_x[pos] = x; }
             total_valid += __popc(bal);
+            finite_entries += __popc(__ballot_sync(kFullMask, finite));
         }
         __syncwarp();
-        int nrow = min(total_valid, k);
-        // Distinct logits can round to one score.  If that happens across the cut between the k-th and
-        // the (k+1)-th entry, cells outside the list may tie with the k-th and precede it by index:
-        // rescan the whole row for the cells with exactly that score, lowest token ids first.
+        // The list is ordered by raw logit, the beam by score, and distinct logits can round to one score.
+        // m = how many list entries compete for the row's k places: k, unless the k-th score continues
+        // past the cut, in which case every entry of that run competes (lowest token ids win).
+        int m = min(total_valid, k);
         if (total_valid > k && tmp_score[k] == tmp_score[k - 1]) {
             const float sb = tmp_score[k - 1];
-            int g = 0;
-            while (g < k && tmp_score[g] > sb) ++g;
-            const int need = k - g;
-            int found = 0;
-            __syncwarp();
-            for (int base = 0; base < V && found < need; base += 32) {
-                const int w = base + lane;
-                bool hit = false;
-                if (w < V) {
-                    const float x = load_logit_dyn(logits, d.dtype, (int64_t)r * stride + w);
-                    hit = x != neg_inf() && !(w == d.eos_id && !eos_ok) && cell_score(x, lse, parent) == sb;
-                }
-                const unsigned bal = __ballot_sync(kFullMask, hit);
-                const int pos = found + __popc(bal & lt_mask);
-                if (hit && pos < need) { tmp_score[g + pos] = sb; tmp_w[g + pos] = w; }
-                found += __popc(bal);
+            int g = k - 1, e = k;
+            while (g > 0 && tmp_score[g - 1] == sb) --g;
+            while (e + 1 < total_valid && tmp_score[e + 1] == sb) ++e;
+            m = e + 1;
+            // If the run reaches the end of a full list, cells outside the list may belong to it.  They
+            // cannot precede the listed ones when the whole run is one logit value (the list holds that
+            // value's lowest ids) and the next lower representable logit already scores below the run.
+            const bool open_end = e == total_valid - 1 && finite_entries == K1;
+            bool rescan = false;
+            if (open_end) {
+                const float xl = tmp_x[e];
+                uint32_t bits = __float_as_uint(xl);
+                const uint32_t ulp = d.dtype == DBA_BF16 ? 0x10000u : 1u;
+                if ((bits << 1) == 0) bits = 0x80000000u | ulp;
+                else bits = (bits & 0x80000000u) ? bits + ulp : bits - ulp;
+                rescan = !(tmp_x[g] == xl && cell_score(__uint_as_float(bits), lse, parent) < sb);
             }
-            __syncwarp();
+            if (rescan) {      // whole row: the cells scoring exactly sb, lowest token ids first
+                const int need = k - g;
+                int found = 0;
+                __syncwarp();
+                for (int base = 0; base < V && found < need; base += 32) {
+                    const int w = base + lane;
+                    bool hit = false;
+                    if (w < V) {
+                        const float x = load_logit_dyn(logits, d.dtype, (int64_t)r * stride + w);
+                        hit = x != neg_inf() && !(w == d.eos_id && !eos_ok) && cell_score(x, lse, parent) == sb;
+                    }
+                    const unsigned bal = __ballot_sync(kFullMask, hit);
+                    const int pos = found + __popc(bal & lt_mask);
+                    if (hit && pos < need) { tmp_score[g + pos] = sb; tmp_w[g + pos] = w; }
+                    found += __popc(bal);
+                }
+                m = k;
+                __syncwarp();
+            }
         }
-        // order by (score desc, token asc) and publish
-        for (int i = lane; i < nrow; i += 32) {
+        // order by (score desc, token asc), keep the first k and publish
+        const int nrow = min(m, k);
+        for (int i = lane; i < m; i += 32) {
             const float si = tmp_score[i]; const int wi = tmp_w[i];
             int rank = 0;
-            for (int j = 0; j < nrow; ++j) rank += cell_better(tmp_score[j], tmp_w[j], si, wi);
-            rt_score[h * k + rank] = si; rt_w[h * k + rank] = wi;
+            for (int j = 0; j < m; ++j) rank += cell_better(tmp_score[j], tmp_w[j], si, wi);
+            if (rank < k) { rt_score[h * k + rank] = si; rt_w[h * k + rank] = wi; }
         }
         if (lane == 0) rt_n[h] = nrow;
         __syncwarp();
@@ -382,10 +406,10 @@ cudaError_t configure_candidates(const Dims& d) {
 cudaError_t launch_candidates(const void* logits, int64_t stride, const Dims& d, const SentCons* cons,
                               const Beam& cur, const ScanOut& part, const float* lse_in, float* row_lse,
                               Cand* cand, int32_t* ncand, int32_t* bank_count, uint32_t* status,
-                              cudaStream_t st, int* launches) {
+                              int32_t* open_count, cudaStream_t st, int* launches) {
     const size_t smem = candidates_smem_bytes(d);
     candidates_kernel<<<d.B, kCandThreads, smem, st>>>(logits, stride, d, cons, cur, part, lse_in, row_lse, cand,
-                                                      ncand, bank_count, status);
+                                                      ncand, bank_count, status, open_count);
     ++*launches;
     return cudaGetLastError();
 }

@@ -25,6 +25,8 @@ struct dba_handle {
     int32_t* ncand;
     int32_t* bank_count;
     uint32_t* status;
+    int32_t* open_list;            // rows the next step scans, and how many
+    int32_t* open_count;
     int32_t* fin_tokens; int32_t* fin_len; float* fin_score; int32_t* fin_flags;
     void* stage_logits;            // only with DBA_FLAG_HOST_STAGING
     dba_step_out stage_out;
@@ -139,6 +141,8 @@ size_t carve(dba_handle* h, void* base, int32_t max_steps) {
     h->ncand = cv.take<int32_t>(d.B);
     h->bank_count = cv.take<int32_t>((size_t)d.B * (kMaxC + 1));
     h->status = cv.take<uint32_t>(64);
+    h->open_list = cv.take<int32_t>(R);
+    h->open_count = cv.take<int32_t>(64);
     h->fin_tokens = cv.take<int32_t>((size_t)d.B * max_steps);
     h->fin_len = cv.take<int32_t>(d.B);
     h->fin_score = cv.take<float>(d.B);
@@ -197,11 +201,12 @@ dba_status dba_init(const dba_config* cfg, void* workspace_dev, size_t workspace
     if (e != cudaSuccess) { delete h; return DBA_ERR_CUDA; }
     if (candidates_smem_bytes(h->d) > (size_t)smem_max) { delete h; return DBA_ERR_UNSUPPORTED; }
     e = configure_candidates(h->d);
+    if (e == cudaSuccess) e = configure_row_scan_tma();
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(h->cons, cons.data(), sizeof(SentCons) * cons.size(), cudaMemcpyHostToDevice, h->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(h->status, 0, 256, h->stream);
     h->launches_tmp = 0;
-    if (e == cudaSuccess) e = launch_reset(h->d, h->beam[0], h->stream, &h->launches_tmp);
+    if (e == cudaSuccess) e = launch_reset(h->d, h->beam[0], h->open_list, h->open_count, h->stream, &h->launches_tmp);
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);   // `cons` is a local buffer
     if (e != cudaSuccess) { delete h; return DBA_ERR_CUDA; }
     h->launches = h->launches_tmp;
@@ -213,7 +218,7 @@ dba_status dba_init(const dba_config* cfg, void* workspace_dev, size_t workspace
 dba_status dba_reset(dba_handle* h) {
     if (!h) return DBA_ERR_INVALID_ARG;
     h->launches_tmp = 0;
-    cudaError_t e = launch_reset(h->d, h->beam[0], h->stream, &h->launches_tmp);
+    cudaError_t e = launch_reset(h->d, h->beam[0], h->open_list, h->open_count, h->stream, &h->launches_tmp);
     h->launches += h->launches_tmp;
     h->t = 0; h->cur = 0;
     return cuda_fail(e);
@@ -243,17 +248,17 @@ dba_status dba_step(dba_handle* h, const void* logits_dev, int64_t row_stride_el
     cudaError_t e = cudaSuccess;
     if (ev) e = cudaEventRecord(ev[0], h->stream);
     if (e == cudaSuccess)
-        e = launch_row_scan(logits_dev, row_stride_elems, h->d, cur.score, cur.token, h->part, h->status,
-                            h->stream, &h->launches_tmp);
+        e = launch_row_scan(logits_dev, row_stride_elems, h->d, cur.score, cur.token, h->open_list, h->open_count,
+                            h->part, h->status, h->sm_count, h->stream, &h->launches_tmp);
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[1], h->stream);
     if (e == cudaSuccess)
         e = launch_candidates(logits_dev, row_stride_elems, h->d, h->cons, cur, h->part, row_lse_in_dev, h->row_lse,
-                              h->cand, h->ncand, h->bank_count, h->status, h->stream, &h->launches_tmp);
+                              h->cand, h->ncand, h->bank_count, h->status, h->open_count, h->stream, &h->launches_tmp);
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[2], h->stream);
     if (e == cudaSuccess)
         e = launch_allocate(h->d, h->cons, cur, nxt, h->cand, h->ncand, h->bank_count, h->row_lse, out,
-                            h->hist_bp + (size_t)h->t * h->d.R, h->hist_tok + (size_t)h->t * h->d.R, h->stream,
-                            &h->launches_tmp);
+                            h->hist_bp + (size_t)h->t * h->d.R, h->hist_tok + (size_t)h->t * h->d.R, h->open_list,
+                            h->open_count, h->stream, &h->launches_tmp);
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[3], h->stream);
     h->launches += h->launches_tmp;
     if (e != cudaSuccess) return DBA_ERR_CUDA;
@@ -396,7 +401,10 @@ dba_status dba_row_scan(const void* logits_dev, int32_t logit_dtype, int32_t R, 
     int launches = 0;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     e = cudaMemsetAsync(status, 0, 256, stream);
-    if (e == cudaSuccess) e = launch_row_scan(logits_dev, row_stride_elems, d, nullptr, nullptr, part, status, stream, &launches);
+    if (e == cudaSuccess) e = configure_row_scan_tma();
+    if (e == cudaSuccess)
+        e = launch_row_scan(logits_dev, row_stride_elems, d, nullptr, nullptr, nullptr, nullptr, part, status, sms, stream,
+                            &launches);
     if (e == cudaSuccess) e = launch_row_merge(d, part, n_top, row_lse_dev, top_val_dev, top_idx_dev, stream, &launches);
     return cuda_fail(e);
 }

@@ -117,23 +117,25 @@ __global__ void row_merge_kernel(int R, int S, int K1, int n_top, const float* _
 }  // namespace
 
 void plan_segments(Dims& d, int sm_count) {
-    // Enough (row, segment) items to occupy every SM a few times over, segments of at least 4096
-    // elements, at most kMaxSeg per row; segment length a multiple of 2048 elements.
-    int S = 1;
-    const int want = 4 * sm_count;
-    while (S < kMaxSeg && d.R * S < want && (d.V + 2 * S - 1) / (2 * S) >= 4096) S *= 2;
-    int seg = (d.V + S - 1) / S;
-    seg = (seg + 2047) / 2048 * 2048;
-    S = (d.V + seg - 1) / seg;
-    d.S = S;
-    d.seg_len = seg;
+    // Segments are 1, 2, 4 or 8 chunks of 8 KB; shorter segments when there are few rows, so that every SM
+    // has several (row, segment) items to work on, but never more than kMaxSeg segments per row.
+    const int es = d.dtype == DBA_F32 ? 4 : 2;
+    const int chunk_elems = 8192 / es;
+    int chunks = 8;
+    auto segs = [&](int c) { return (d.V + c * chunk_elems - 1) / (c * chunk_elems); };
+    while (segs(chunks) > kMaxSeg) chunks *= 2;                       // very long rows: longer segments
+    while (chunks > 1 && (int64_t)d.R * segs(chunks) < 6LL * sm_count && segs(chunks / 2) <= kMaxSeg) chunks /= 2;
+    d.seg_len = chunks * chunk_elems;
+    d.S = segs(chunks);
     d.K1 = d.k + 2;
 }
 
 cudaError_t launch_row_scan(const void* logits, int64_t stride, const Dims& d, const float* open_score,
-                            const int32_t* open_token, const ScanOut& out, uint32_t* status,
-                            cudaStream_t st, int* launches) {
-    (void)status;
+                            const int32_t* open_token, const int32_t* open_list, const int32_t* open_count,
+                            const ScanOut& out, uint32_t* status, int sm_count, cudaStream_t st, int* launches) {
+    ++*launches;
+    if (row_scan_tma_usable(logits, stride, d))
+        return launch_row_scan_tma(logits, stride, d, open_list, open_count, out, status, sm_count, st);
     const int items = d.R * d.S;
     if (d.dtype == DBA_F32)
         row_scan_generic_kernel<float><<<items, kScanThreads, 0, st>>>(
@@ -143,7 +145,6 @@ cudaError_t launch_row_scan(const void* logits, int64_t stride, const Dims& d, c
         row_scan_generic_kernel<__nv_bfloat16><<<items, kScanThreads, 0, st>>>(
             (const __nv_bfloat16*)logits, stride, d.V, d.S, d.seg_len, d.K1, d.eos_id, open_score, open_token,
             out.m, out.s, out.top_val, out.top_idx);
-    ++*launches;
     return cudaGetLastError();
 }
 
