@@ -1,16 +1,22 @@
 // Row scan, streaming version for sm_100a: one HBM pass per row.
 //
-// A persistent CTA per SM works through (row, segment) items.  Three roles, all synchronised with mbarriers:
-//   producer   one thread issues bulk asynchronous copies (TMA, cp.async.bulk) of 8 KB chunks of the row into
-//              a ring of shared-memory stages;
-//   consumers  stream every chunk once: exp2 of (x - reference) summed per lane (Section 2's normaliser), and
-//              a per-lane running maximum; no selection logic in this loop;
-//   selectors  one item behind: from the consumers' lane maxima they take a lower bound of the K1-th largest
-//              entry (the K1-th largest of 256 disjoint group maxima is one), pass over the item's chunks
-//              again while they are still in shared memory, collect the few entries at or above the bound,
-//              order them exactly (value descending, lower index first) and write the segment's partial
-//              result; only then are the stages handed back to the producer.
+// A persistent CTA per SM works through (row, segment) items; a segment is up to eight 8 KB chunks.  Warps have
+// fixed roles and talk through mbarriers only (no CTA-wide barrier inside the loop):
+//   producer    one thread issues bulk asynchronous copies (TMA, cp.async.bulk) of the chunks into a ring of
+//               shared-memory stages;
+//   consumers   each warp streams half a chunk of the item: the maximum first, then exp2(x*log2e - c) summed per
+//               lane (Section 2's normaliser) with c a whole number at or above the maximum; it leaves one
+//               maximum per lane; no selection logic in this loop;
+//   bound       one warp turns the lane maxima into a lower bound of the K1-th largest entry of the item: the
+//               K1-th largest of maxima of disjoint groups is one; found exactly by bisection on ordered keys;
+//   pass B      warps look again only at the vectors of lanes whose maximum reaches the bound (a few dozen of
+//               the 4096 vectors of an item), collect the entries at or above the bound, and hand the stages
+//               back to the producer;
+//   ranking     one warp orders the collected entries exactly (value descending, lower index first) and
+//               writes the segment's partial result.
 // Every wait is bounded: a wait that runs out sets the timeout bit of the status word and the CTA winds down.
+// The code is kept small on purpose: the roles run different code at the same time and share one
+// instruction cache.
 #include <cuda_bf16.h>
 
 #include "dba_device.cuh"
@@ -21,35 +27,38 @@ namespace dba {
 namespace {
 
 constexpr int kChunkBytes = 8192;
-constexpr int kStages = 24;                 // 192 KB of ring
-constexpr int kMaxSegChunks = 8;            // a segment is at most 64 KB
-constexpr int kNC = 8;                      // consumer warps
-constexpr int kNS = 4;                      // selector warps
-constexpr int kThreads = 32 * (1 + kNC + kNS);
-constexpr int kConsThreads = 32 * kNC;
-constexpr int kSelThreads = 32 * kNS;
-constexpr int kSlots = 4;                   // items whose lane maxima may be pending at once
-constexpr int kCandCap = 1024;              // entries at or above the bound that one item may hold
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kChunkVecs = kChunkBytes / 16;   // 512
+constexpr int kHalfVecs = kChunkVecs / 2;      // vectors of half a chunk: 8 per lane
+constexpr int kVecsPerLane = kHalfVecs / 32;   // 8
+constexpr int kStages = 24;                    // 192 KB of ring
+constexpr int kMaxSegChunks = 8;               // a segment is at most 64 KB
+constexpr int kNC = 2 * kMaxSegChunks;         // consumer warps, half a chunk of the item each
+constexpr int kNS = 4;                         // pass-B warps, two chunks of the item each
+constexpr int kWarpBound = 1 + kNC;            // warp index of the bound warp
+constexpr int kWarpPassB = kWarpBound + 1;     // first pass-B warp
+constexpr int kWarpRank = kWarpPassB + kNS;    // ranking warp
+constexpr int kThreads = 32 * (kWarpRank + 1);
+constexpr int kSlots = 4;                      // items in flight between consumers and ranking
+constexpr int kCandCap = 256;                  // entries at or above the bound that one item may hold
+constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr uint32_t kSuspendHint = 0x989680u;   // lets a waiting thread sleep in hardware until the phase completes
 constexpr float kLog2e = 1.44269502162933349609375f;        // fl32(log2(e))
-constexpr double kLn2 = 0.69314718055994530942;
 
 struct Smem {
     alignas(128) unsigned char ring[kStages][kChunkBytes];
     alignas(8) uint64_t full[kStages];
     uint64_t empty[kStages];
     uint64_t item_done[kSlots];
+    uint64_t bound_ready[kSlots];
+    uint64_t passb_done[kSlots];
     uint64_t slot_free[kSlots];
-    uint64_t cand[kCandCap];
-    float lane_max[kSlots][kConsThreads];
+    uint64_t cand[kSlots][kCandCap];
+    float lane_max[kSlots][kNC][32];
     float warp_sum[kSlots][kNC];
-    float warp_ref[kSlots][kNC];            // the constant c of exp2(x*log2e - c) each warp ended with
-    int hist1[256];
-    int hist2[256];
-    int sel_b1, sel_rank, sel_thr_ord;
-    int cand_count;
+    float warp_ref[kSlots][kNC];            // the whole number c of exp2(x*log2e - c) each warp used (-inf: no data)
+    float bound_lo[kSlots];                 // entries >= bound_lo are collected
+    int cand_count[kSlots];                 // above kCandCap: the list overflowed
     int abort_flag;
-    uint64_t red[kNS];
 };
 
 struct Params {
@@ -76,75 +85,148 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHint) : "memory");
     return ok != 0;
 }
 // Bounded wait.  Returns false when the CTA is winding down (this wait ran out, or another one did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 255u && *abort_flag) return false;
+        if (*abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
+}
+// The same for a whole warp (every lane observes the phase itself); the answer is the same on all lanes.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    bool ok = mbar_try_wait(bar, parity);
+    if (!ok) ok = mbar_wait(bar, parity, abort_flag);
+    return __all_sync(kFullMask, ok);
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void sel_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kSelThreads) : "memory"); }
-// Barrier of the selector group that also ORs a flag over its threads: every thread gets the same answer.
-__device__ __forceinline__ bool sel_barrier_or(int flag) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.s32 q, %1, 0;\n\tbar.red.or.pred p, 1, %2, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(r) : "r"(flag), "n"(kSelThreads) : "memory");
-    return r != 0;
-}
 __device__ __forceinline__ float ex2(float t) { float r; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t)); return r; }
+// 2^d for an integer d <= 0, exact (0 below the normal range)
+__device__ __forceinline__ float pow2i(int d) { return d < -126 ? 0.f : __int_as_float((d + 127) << 23); }
 __device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
     uint32_t r; asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b)); return r;
 }
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+// two fp32 values in one 64-bit register, for the packed fma / add of sm_100
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) { uint64_t d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) { uint64_t d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+// acc += (2^(a*L + C), 2^(b*L + C)) for packed constants L2 = (L, L), C2 = (C, C)
+__device__ __forceinline__ uint64_t exp_acc(uint64_t acc, float a, float b, uint64_t L2, uint64_t C2) {
+    float t0, t1;
+    unpack2(fma2(pack2(a, b), L2, C2), t0, t1);
+    return add2(acc, pack2(ex2(t0), ex2(t1)));
+}
 
 template <typename T> struct Vec;
 template <> struct Vec<float> {
     static constexpr int kElems = 4;
-    static __device__ __forceinline__ float vmax(const uint4& v) {
-        return fmaxf(fmaxf(__uint_as_float(v.x), __uint_as_float(v.y)), fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
+    static constexpr uint32_t kNegInfWord = 0xff800000u;
+    // running maximum of vectors, kept in a form that is cheap to update
+    typedef float Max;
+    static __device__ __forceinline__ Max max_init() { return neg_inf(); }
+    static __device__ __forceinline__ Max max_update(Max m, const uint4& v) {
+        return fmaxf(fmaxf(m, fmaxf(__uint_as_float(v.x), __uint_as_float(v.y))), fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
     }
+    static __device__ __forceinline__ float max_value(Max m) { return m; }
     static __device__ __forceinline__ void unpack(const uint4& v, float* x) {
         x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y); x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+    }
+    static __device__ __forceinline__ void exp_sum(const uint4& v, uint64_t L2, uint64_t C2, uint64_t& a0, uint64_t& a1) {
+        a0 = exp_acc(a0, __uint_as_float(v.x), __uint_as_float(v.y), L2, C2);
+        a1 = exp_acc(a1, __uint_as_float(v.z), __uint_as_float(v.w), L2, C2);
     }
 };
 template <> struct Vec<__nv_bfloat16> {
     static constexpr int kElems = 8;
-    static __device__ __forceinline__ float vmax(const uint4& v) {
-        const uint32_t m = max_bf16x2(max_bf16x2(v.x, v.y), max_bf16x2(v.z, v.w));
-        return fmaxf(bf16_lo(m), bf16_hi(m));
+    static constexpr uint32_t kNegInfWord = 0xff80ff80u;
+    typedef uint32_t Max;       // two bf16 maxima
+    static __device__ __forceinline__ Max max_init() { return kNegInfWord; }
+    static __device__ __forceinline__ Max max_update(Max m, const uint4& v) {
+        return max_bf16x2(max_bf16x2(m, max_bf16x2(v.x, v.y)), max_bf16x2(v.z, v.w));
     }
+    static __device__ __forceinline__ float max_value(Max m) { return fmaxf(bf16_lo(m), bf16_hi(m)); }
     static __device__ __forceinline__ void unpack(const uint4& v, float* x) {
         x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2] = bf16_lo(v.y); x[3] = bf16_hi(v.y);
         x[4] = bf16_lo(v.z); x[5] = bf16_hi(v.z); x[6] = bf16_lo(v.w); x[7] = bf16_hi(v.w);
     }
+    static __device__ __forceinline__ void exp_sum(const uint4& v, uint64_t L2, uint64_t C2, uint64_t& a0, uint64_t& a1) {
+        a0 = exp_acc(a0, bf16_lo(v.x), bf16_hi(v.x), L2, C2);
+        a1 = exp_acc(a1, bf16_lo(v.y), bf16_hi(v.y), L2, C2);
+        a0 = exp_acc(a0, bf16_lo(v.z), bf16_hi(v.z), L2, C2);
+        a1 = exp_acc(a1, bf16_lo(v.w), bf16_hi(v.w), L2, C2);
+    }
 };
 
-// Walks the items of this CTA in the order all three roles agree on.
+// The items of this CTA, in the order all roles agree on, with the ring position of each item's first chunk.
+// Items are numbered row-major over (position in the list of open rows, segment); this CTA takes every
+// gridDim.x-th one.  The walk needs no division after the constructor.
 struct ItemIter {
-    int item, n_items, S;
+    int i, seg_, n_rows, S, step_i, step_seg, seg_bytes_full, row_bytes;
+    int row_, bytes_, n_chunks_;        // of the current item
+    uint32_t fills, n_item;
     const int32_t* open_list;
-    __device__ ItemIter(const Params& p) : S(p.S), open_list(p.open_list) {
-        const int rows = p.open_count ? *p.open_count : p.R;
-        n_items = rows * p.S;
-        item = blockIdx.x;
+    __device__ ItemIter(const Params& p, int elem_bytes) : S(p.S), fills(0), n_item(0), open_list(p.open_list) {
+        n_rows = p.open_count ? *p.open_count : p.R;
+        i = blockIdx.x / S; seg_ = blockIdx.x - i * S;
+        step_i = gridDim.x / S; step_seg = gridDim.x - step_i * S;
+        seg_bytes_full = p.seg_len * elem_bytes;
+        row_bytes = p.V * elem_bytes;
+        load();
     }
-    __device__ bool valid() const { return item < n_items; }
-    __device__ void next() { item += gridDim.x; }
-    __device__ int row() const { const int i = item / S; return open_list ? open_list[i] : i; }
-    __device__ int seg() const { return item % S; }
+    __device__ __forceinline__ void load() {
+        if (i >= n_rows) return;
+        row_ = open_list ? open_list[i] : i;
+        bytes_ = min(seg_bytes_full, row_bytes - seg_ * seg_bytes_full);
+        n_chunks_ = (bytes_ + kChunkBytes - 1) / kChunkBytes;
+    }
+    __device__ bool valid() const { return i < n_rows; }
+    __device__ void next() {
+        fills += (uint32_t)n_chunks_; n_item += 1;
+        i += step_i; seg_ += step_seg;
+        if (seg_ >= S) { seg_ -= S; ++i; }
+        load();
+    }
+    __device__ int row() const { return row_; }
+    __device__ int seg() const { return seg_; }
+    __device__ int bytes() const { return bytes_; }
+    __device__ int n_chunks() const { return n_chunks_; }
+    __device__ uint32_t slot() const { return n_item % kSlots; }
+    __device__ uint32_t slot_phase() const { return (n_item / kSlots) & 1u; }
+    __device__ uint32_t stage(int c) const { return (fills + (uint32_t)c) % kStages; }
+    __device__ uint32_t stage_phase(int c) const { return ((fills + (uint32_t)c) / kStages) & 1u; }
+    __device__ int chunk_vecs(int c) const { return min(kChunkBytes, bytes_ - c * kChunkBytes) >> 4; }
 };
+
+// Ranking, rare path: more entries at or above the bound than the list holds (long runs of equal values at the
+// bound, or an adversarial layout): take the K1 best one at a time, reading the segment again from global memory.
+template <typename T>
+__device__ __noinline__ void rank_from_global(const T* src, int e0, int e1, int K1, float* tv, int32_t* ti) {
+    const int lane = threadIdx.x & 31;
+    uint64_t prev = ~0ull;
+#pragma unroll 1
+    for (int r2 = 0; r2 < K1; ++r2) {
+        uint64_t best = 0;
+#pragma unroll 2
+        for (int w = e0 + lane; w < e1; w += 32) {
+            const uint64_t kk = row_key(load_logit<T>(src + w), w);
+            if (kk < prev && kk > best) best = kk;
+        }
+        best = warp_max_u64(best);
+        if (lane == 0) { tv[r2] = best ? row_key_val(best) : neg_inf(); ti[r2] = best ? row_key_idx(best) : -1; }
+        prev = best;      // 0 once exhausted: nothing is below it
+    }
+}
 
 template <typename T>
 __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
@@ -152,264 +234,229 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
     Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
     constexpr int kElems = Vec<T>::kElems;
     constexpr int kChunkElems = kChunkBytes / (int)sizeof(T);
-    constexpr int kChunkVecs = kChunkBytes / 16;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     volatile int* abort_flag = &sm.abort_flag;
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sm.full[s]), 1); mbar_init(smem_u32(&sm.empty[s]), kNS); }
-        for (int s = 0; s < kSlots; ++s) { mbar_init(smem_u32(&sm.item_done[s]), kNC); mbar_init(smem_u32(&sm.slot_free[s]), 1); }
-        sm.cand_count = 0; sm.abort_flag = 0;
+        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sm.full[s]), 1); mbar_init(smem_u32(&sm.empty[s]), 1); }
+        for (int s = 0; s < kSlots; ++s) {
+            mbar_init(smem_u32(&sm.item_done[s]), kNC); mbar_init(smem_u32(&sm.bound_ready[s]), 1);
+            mbar_init(smem_u32(&sm.passb_done[s]), kNS); mbar_init(smem_u32(&sm.slot_free[s]), 1);
+            sm.cand_count[s] = 0;
+        }
+        sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = tid; i < 256; i += kThreads) { sm.hist1[i] = 0; sm.hist2[i] = 0; }
     __syncthreads();
-
-    const int seg_bytes_full = p.seg_len * (int)sizeof(T);
-    const int row_bytes = p.V * (int)sizeof(T);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            uint32_t fills = 0;
+            ItemIter it(p, (int)sizeof(T));
             bool ok = true;
-            for (ItemIter it(p); ok && it.valid(); it.next()) {
-                const int seg = it.seg();
-                const char* src = (const char*)p.logits + ((int64_t)it.row() * p.stride + (int64_t)seg * p.seg_len) * (int64_t)sizeof(T);
-                int left = min(seg_bytes_full, row_bytes - seg * seg_bytes_full);
-                while (left > 0) {
-                    const int bytes = min(left, kChunkBytes);
-                    const uint32_t st = fills % kStages, ph = (fills / kStages) & 1u;
-                    if (!mbar_wait(smem_u32(&sm.empty[st]), ph ^ 1u, abort_flag)) { ok = false; break; }
-                    mbar_expect_tx(smem_u32(&sm.full[st]), (uint32_t)bytes);
-                    bulk_load(smem_u32(sm.ring[st]), src, (uint32_t)bytes, smem_u32(&sm.full[st]));
-                    src += bytes; left -= bytes; ++fills;
+#pragma unroll 1
+            for (; ok && it.valid(); it.next()) {
+                const char* src = (const char*)p.logits + ((int64_t)it.row() * p.stride + (int64_t)it.seg() * p.seg_len) * (int64_t)sizeof(T);
+                const int nc = it.n_chunks();
+#pragma unroll 1
+                for (int c = 0; c < nc; ++c) {
+                    const uint32_t st = it.stage(c);
+                    if (!mbar_try_wait(smem_u32(&sm.empty[st]), it.stage_phase(c) ^ 1u) &&
+                        !mbar_wait(smem_u32(&sm.empty[st]), it.stage_phase(c) ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t bytes = (uint32_t)it.chunk_vecs(c) << 4;
+                    mbar_expect_tx(smem_u32(&sm.full[st]), bytes);
+                    bulk_load(smem_u32(sm.ring[st]), src + (int64_t)c * kChunkBytes, bytes, smem_u32(&sm.full[st]));
                 }
             }
             if (!ok) {   // winding down: let the copies already issued land before the CTA leaves
+                const uint32_t fills = it.fills + kMaxSegChunks;
                 const uint32_t first = fills > kStages ? fills - kStages : 0;
-                for (uint32_t f = first; f < fills; ++f) {
-                    const uint32_t st = f % kStages, ph = (f / kStages) & 1u;
-                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&sm.full[st]), ph); ++i) {}
-                }
+#pragma unroll 1
+                for (uint32_t f = first; f < fills; ++f)
+                    for (uint32_t i = 0; i < 64 && !mbar_try_wait(smem_u32(&sm.full[f % kStages]), (f / kStages) & 1u); ++i) {}
             }
         }
         __syncwarp();
     } else if (warp <= kNC) {
         // ------------------------------------------------------------------ consumers
-        const int cw = warp - 1, ctid = cw * 32 + lane;
-        uint32_t fills = 0, n_item = 0;
-        bool ok = true;
-        for (ItemIter it(p); ok && it.valid(); it.next(), ++n_item) {
-            const int seg = it.seg();
-            const int bytes_item = min(seg_bytes_full, row_bytes - seg * seg_bytes_full);
-            const uint32_t slot = n_item % kSlots, slot_ph = (n_item / kSlots) & 1u;
-            float ssum = 0.f, lmax = neg_inf();
-            float ref = 0.f, negc = 0.f;          // exp2(x*log2e + negc); ref = the value negc was made from
-            bool have_ref = false;
-            for (int done = 0; done < bytes_item; done += kChunkBytes, ++fills) {
-                const int bytes = min(kChunkBytes, bytes_item - done);
-                const uint32_t st = fills % kStages, ph = (fills / kStages) & 1u;
-                if (!__all_sync(kFullMask, mbar_wait(smem_u32(&sm.full[st]), ph, abort_flag))) { ok = false; break; }
-                const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[st]);
-                const int nvec = bytes >> 4;
-                uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
-                const bool h0 = ctid < nvec, h1 = ctid + kConsThreads < nvec;
-                if (h0) v0 = vec[ctid];
-                if (h1) v1 = vec[ctid + kConsThreads];
-                float m2 = neg_inf();
-                if (h0) m2 = Vec<T>::vmax(v0);
-                if (h1) m2 = fmaxf(m2, Vec<T>::vmax(v1));
-                lmax = fmaxf(lmax, m2);
-                // keep the exponent argument well inside fp32 range: move the reference up when needed
-                if (__any_sync(kFullMask, have_ref ? m2 > ref + 32.f : m2 > neg_inf())) {
-                    float nm = warp_max(m2);
-                    if (have_ref) { nm = fmaxf(nm, ref); ssum *= ex2((ref - nm) * kLog2e); }
-                    ref = nm; negc = -(nm * kLog2e); have_ref = true;
-                }
-                float x[kElems];
-                if (h0) {
-                    Vec<T>::unpack(v0, x);
+        const int cw = warp - 1, chunk = cw >> 1, half = cw & 1;
+#pragma unroll 1
+        for (ItemIter it(p, (int)sizeof(T)); it.valid(); it.next()) {
+            float lmax = neg_inf(), ssum = 0.f, cref = neg_inf();
+            const int nvec = chunk < it.n_chunks() ? it.chunk_vecs(chunk) - half * kHalfVecs : 0;
+            if (nvec > 0) {
+                if (!mbar_wait_warp(smem_u32(&sm.full[it.stage(chunk)]), it.stage_phase(chunk), abort_flag)) break;
+                const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[it.stage(chunk)]) + half * kHalfVecs + lane;
+                uint4 v[kVecsPerLane];
+                if (nvec >= kHalfVecs) {
 #pragma unroll
-                    for (int e = 0; e < kElems; ++e) ssum += ex2(fmaf(x[e], kLog2e, negc));
-                }
-                if (h1) {
-                    Vec<T>::unpack(v1, x);
+                    for (int i = 0; i < kVecsPerLane; ++i) v[i] = vec[i * 32];
+                } else {
 #pragma unroll
-                    for (int e = 0; e < kElems; ++e) ssum += ex2(fmaf(x[e], kLog2e, negc));
-                }
-            }
-            if (!ok) break;
-            // hand the lane maxima and the warp's sum to the selectors
-            if (!__all_sync(kFullMask, mbar_wait(smem_u32(&sm.slot_free[slot]), slot_ph ^ 1u, abort_flag))) break;
-            sm.lane_max[slot][ctid] = lmax;
-            const float wsum = warp_sum(ssum);
-            if (lane == 0) { sm.warp_sum[slot][cw] = wsum; sm.warp_ref[slot][cw] = -negc; }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sm.item_done[slot]));
-        }
-    } else {
-        // ------------------------------------------------------------------ selectors
-        const int sw = warp - 1 - kNC, stid = sw * 32 + lane;
-        uint32_t fills = 0, n_item = 0;
-        bool ok = true;
-        for (ItemIter it(p); ok && it.valid(); it.next(), ++n_item) {
-            const int row = it.row(), seg = it.seg();
-            const int bytes_item = min(seg_bytes_full, row_bytes - seg * seg_bytes_full);
-            const uint32_t slot = n_item % kSlots, slot_ph = (n_item / kSlots) & 1u;
-            const int64_t out = (int64_t)row * p.S + seg;
-            mbar_wait(smem_u32(&sm.item_done[slot]), slot_ph, abort_flag);
-            if (sel_barrier_or(*abort_flag)) { ok = false; break; }      // one answer for the whole group
-
-            // ---- bound: the K1-th largest of the 256 lane maxima, to 16 bits of the ordered key ----
-            uint32_t key[kConsThreads / kSelThreads];
-#pragma unroll
-            for (int q = 0; q < kConsThreads / kSelThreads; ++q) {
-                key[q] = ord32(sm.lane_max[slot][stid + q * kSelThreads]);
-                atomicAdd(&sm.hist1[key[q] >> 24], 1);
-            }
-            if (stid == 0) {   // the segment's normaliser parts, combined in double
-                double C = -1e300;
-                for (int w = 0; w < kNC; ++w) C = fmax(C, (double)sm.warp_ref[slot][w]);
-                double S = 0.0;
-                for (int w = 0; w < kNC; ++w) S += (double)sm.warp_sum[slot][w] * exp2((double)sm.warp_ref[slot][w] - C);
-                // sum_x 2^(x*log2e) = S * 2^C  ->  (m, s) with sum_x e^x = s * e^m
-                float m = (float)(C * kLn2);
-                float s = (float)(S * exp(C * kLn2 - (double)m));
-                if (S == 0.0) { m = neg_inf(); s = 0.f; }
-                p.part_m[out] = m; p.part_s[out] = s;
-            }
-            sel_barrier();
-            if (sw == 0) {     // highest 8-bit digit whose suffix count reaches K1
-                int c[8], tot = 0;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { c[j] = sm.hist1[lane * 8 + j]; tot += c[j]; }
-                int suf = tot;                                  // inclusive suffix over lanes
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_down_sync(kFullMask, suf, o); if (lane + o < 32) suf += t; }
-                const int above = suf - tot;                    // count in lanes above this one
-                int run = above, b1 = -1, rank = 0;
-#pragma unroll
-                for (int j = 7; j >= 0; --j) { if (b1 < 0 && run + c[j] >= p.K1) { b1 = lane * 8 + j; rank = p.K1 - run; } run += c[j]; }
-                const unsigned hit = __ballot_sync(kFullMask, b1 >= 0);
-                const int src = hit ? 31 - __clz(hit) : 0;      // the highest lane that found it
-                b1 = __shfl_sync(kFullMask, b1, src); rank = __shfl_sync(kFullMask, rank, src);
-                if (lane == 0) { sm.sel_b1 = hit ? b1 : 0; sm.sel_rank = hit ? rank : 1; }
-#pragma unroll
-                for (int j = 0; j < 8; ++j) sm.hist1[lane * 8 + j] = 0;
-            }
-            sel_barrier();
-            const int b1 = sm.sel_b1;
-#pragma unroll
-            for (int q = 0; q < kConsThreads / kSelThreads; ++q)
-                if ((int)(key[q] >> 24) == b1) atomicAdd(&sm.hist2[(key[q] >> 16) & 255u], 1);
-            sel_barrier();
-            if (sw == 0) {
-                const int want = sm.sel_rank;
-                int c[8], tot = 0;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { c[j] = sm.hist2[lane * 8 + j]; tot += c[j]; }
-                int suf = tot;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_down_sync(kFullMask, suf, o); if (lane + o < 32) suf += t; }
-                int run = suf - tot, b2 = -1;
-#pragma unroll
-                for (int j = 7; j >= 0; --j) { if (b2 < 0 && run + c[j] >= want) b2 = lane * 8 + j; run += c[j]; }
-                const unsigned hit = __ballot_sync(kFullMask, b2 >= 0);
-                const int src = hit ? 31 - __clz(hit) : 0;
-                b2 = __shfl_sync(kFullMask, b2, src);
-                if (lane == 0) sm.sel_thr_ord = (int)(((uint32_t)b1 << 24) | ((uint32_t)(hit ? b2 : 0) << 16));
-#pragma unroll
-                for (int j = 0; j < 8; ++j) sm.hist2[lane * 8 + j] = 0;
-            }
-            sel_barrier();
-            float thr = unord32((uint32_t)sm.sel_thr_ord);
-            if (!(thr == thr)) thr = neg_inf();          // the bucket that holds -inf has no finite lower edge
-            // the consumers may reuse this slot from here on
-            if (stid == 0) mbar_arrive(smem_u32(&sm.slot_free[slot]));
-
-            // ---- second look at the item's chunks: everything at or above the bound ----
-            const int elem0 = seg * p.seg_len;
-            int chunk = 0;
-            for (int done = 0; done < bytes_item; done += kChunkBytes, ++fills, ++chunk) {
-                const int bytes = min(kChunkBytes, bytes_item - done);
-                const uint32_t st = fills % kStages, ph = (fills / kStages) & 1u;
-                mbar_wait(smem_u32(&sm.full[st]), ph, abort_flag);   // complete already: the consumers waited on it
-                const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[st]);
-                const int nvec = bytes >> 4;
-#pragma unroll
-                for (int q = 0; q < kChunkVecs / kSelThreads; ++q) {
-                    const int vi = stid + q * kSelThreads;
-                    if (vi < nvec) {
-                        const uint4 v = vec[vi];
-                        if (Vec<T>::vmax(v) >= thr) {
-                            float x[kElems];
-                            Vec<T>::unpack(v, x);
-                            const int base = elem0 + chunk * kChunkElems + vi * kElems;
-#pragma unroll
-                            for (int e = 0; e < kElems; ++e)
-                                if (x[e] >= thr) {
-                                    const int pos = atomicAdd(&sm.cand_count, 1);
-                                    if (pos < kCandCap) sm.cand[pos] = row_key(x[e], base + e);
-                                }
-                        }
+                    for (int i = 0; i < kVecsPerLane; ++i) {
+                        const uint32_t w = Vec<T>::kNegInfWord;
+                        v[i] = i * 32 + lane < nvec ? vec[i * 32] : make_uint4(w, w, w, w);   // beyond the row: -inf
                     }
                 }
+                typename Vec<T>::Max pm = Vec<T>::max_init();
+#pragma unroll
+                for (int i = 0; i < kVecsPerLane; ++i) pm = Vec<T>::max_update(pm, v[i]);
+                lmax = Vec<T>::max_value(pm);
+                const float wm = warp_max(lmax);
+                if (wm != neg_inf()) {
+                    cref = ceilf(wm * kLog2e);            // a whole number: rescaling by powers of two is exact
+                    const uint64_t L2 = pack2(kLog2e, kLog2e), C2 = pack2(-cref, -cref);
+                    uint64_t a0 = 0, a1 = 0;
+#pragma unroll
+                    for (int i = 0; i < kVecsPerLane; ++i) Vec<T>::exp_sum(v[i], L2, C2, a0, a1);
+                    float s0, s1, s2, s3;
+                    unpack2(a0, s0, s1); unpack2(a1, s2, s3);
+                    ssum = (s0 + s1) + (s2 + s3);
+                }
             }
-            sel_barrier();       // the stages are released below, once it is known whether they are still needed
-            const int n = sm.cand_count;
-            const uint32_t fills_end = fills;
-            const int n_chunks = chunk;
+            // hand the lane maxima and the warp's sum over
+            if (!mbar_wait_warp(smem_u32(&sm.slot_free[it.slot()]), it.slot_phase() ^ 1u, abort_flag)) break;
+            sm.lane_max[it.slot()][cw][lane] = lmax;
+            const float wsum = warp_sum(ssum);
+            if (lane == 0) { sm.warp_sum[it.slot()][cw] = wsum; sm.warp_ref[it.slot()][cw] = cref; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm.item_done[it.slot()]));
+        }
+    } else if (warp == kWarpBound) {
+        // ------------------------------------------------------------------ bound
+#pragma unroll 1
+        for (ItemIter it(p, (int)sizeof(T)); it.valid(); it.next()) {
+            const uint32_t slot = it.slot();
+            if (!mbar_wait_warp(smem_u32(&sm.item_done[slot]), it.slot_phase(), abort_flag)) break;
+            // K1-th largest of 256 group maxima (a group = the two lanes that share a chunk position), exactly,
+            // by bisection on their ordered keys (bf16 values need 16 key bits, fp32 values 32); the bits all
+            // keys share are skipped
+            constexpr int kKeyBits = sizeof(T) == 2 ? 16 : 32;
+            constexpr int kGroups = kNC / 2;
+            uint32_t key[kGroups], orv = 0, andv = ~0u;
+#pragma unroll
+            for (int w = 0; w < kGroups; ++w) {
+                key[w] = ord32(fmaxf(sm.lane_max[slot][2 * w][lane], sm.lane_max[slot][2 * w + 1][lane])) >> (32 - kKeyBits);
+                orv |= key[w]; andv &= key[w];
+            }
+            orv = __reduce_or_sync(kFullMask, orv); andv = __reduce_and_sync(kFullMask, andv);
+            uint32_t t = andv;
+            if (orv != andv) {
+                const int top = 31 - __clz(orv ^ andv);
+                t = andv & ~((2u << top) - 1u);
+#pragma unroll 1
+                for (int bit = top; bit >= 0; --bit) {
+                    const uint32_t c = t | (1u << bit);
+                    int cnt = 0;
+#pragma unroll
+                    for (int w = 0; w < kGroups; ++w) cnt += key[w] >= c;
+                    if ((int)__reduce_add_sync(kFullMask, cnt) >= p.K1) t = c;
+                }
+            }
+            if (lane == 0) {
+                uint32_t o = t;
+                if (kKeyBits == 16) o = (t << 16) | ((t & 0x8000u) ? 0u : 0xffffu);   // a bf16 value's low key bits
+                sm.bound_lo[slot] = unord32(o);      // an actual lane maximum (possibly -inf)
+                // the segment's normaliser: sum_x 2^(x*log2e) = S * 2^C with a whole number C
+                float C = neg_inf();
+#pragma unroll 1
+                for (int w = 0; w < kNC; ++w) C = fmaxf(C, sm.warp_ref[slot][w]);
+                float m = neg_inf(), s2 = 0.f;
+                if (C != neg_inf()) {
+                    float S = 0.f;
+#pragma unroll 1
+                    for (int w = 0; w < kNC; ++w) {
+                        const float cw2 = sm.warp_ref[slot][w];
+                        if (cw2 != neg_inf()) S += sm.warp_sum[slot][w] * pow2i((int)(cw2 - C));
+                    }
+                    // (m, s) with sum_x e^x = s * e^m: m = fl32(C ln2), the rounding of m folded into s
+                    constexpr float kLn2Hi = 0.693147182464599609375f, kLn2Lo = -1.904654299957767e-9f;
+                    m = C * kLn2Hi;
+                    const float err = fmaf(C, kLn2Hi, -m) + C * kLn2Lo;
+                    s2 = fmaf(S, err, S);
+                }
+                const int64_t out = (int64_t)it.row() * p.S + it.seg();
+                p.part_m[out] = m; p.part_s[out] = s2;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm.bound_ready[slot]));
+        }
+    } else if (warp < kWarpRank) {
+        // ------------------------------------------------------------------ pass B
+        // This warp owns consumer warps 4*sw .. 4*sw+3, i.e. chunks 2*sw and 2*sw+1 of every item.  Only lanes
+        // whose maximum reaches the bound can hold an entry at or above it; up to four such lanes are handled
+        // at a time, eight lanes of this warp looking at the eight vectors of one of them.
+        const int sw = warp - kWarpPassB, grp = lane >> 3, vrow = lane & 7;
+#pragma unroll 1
+        for (ItemIter it(p, (int)sizeof(T)); it.valid(); it.next()) {
+            const uint32_t slot = it.slot();
+            if (!mbar_wait_warp(smem_u32(&sm.bound_ready[slot]), it.slot_phase(), abort_flag)) break;
+            // The chunks' bytes are visible here: their consumers observed the copies' completion before they
+            // reported the item done, and that report is ordered before the bound this warp has just waited for.
+            const float lo = sm.bound_lo[slot];
+            const int nc = it.n_chunks();
+            const int elem0 = it.seg() * p.seg_len;
+#pragma unroll 1
+            for (int q = 0; q < 4; ++q) {
+                const int w = 4 * sw + q, chunk = w >> 1, half = w & 1;
+                if (chunk >= nc) break;
+                unsigned m = __ballot_sync(kFullMask, sm.lane_max[slot][w][lane] >= lo);
+                const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[it.stage(chunk)]);
+                const int nvec = it.chunk_vecs(chunk);
+                while (m) {
+                    unsigned mm = m;                                   // the grp-th lowest set bit, if there is one
+                    for (int j = 0; j < grp; ++j) mm &= mm - 1;
+                    const int src_lane = __ffs(mm) - 1;
+                    const int vi = half * kHalfVecs + vrow * 32 + src_lane;
+                    if (mm && vi < nvec) {
+                        float x[kElems];
+                        Vec<T>::unpack(vec[vi], x);
+                        const int base = elem0 + chunk * kChunkElems + vi * kElems;
+#pragma unroll
+                        for (int e = 0; e < kElems; ++e)
+                            if (x[e] >= lo) {
+                                const int pos = atomicAdd(&sm.cand_count[slot], 1);
+                                if (pos < kCandCap) sm.cand[slot][pos] = row_key(x[e], base + e);
+                            }
+                    }
+                    m &= m - 1; m &= m - 1; m &= m - 1; m &= m - 1;     // four lanes done
+                    __syncwarp();
+                }
+            }
+            __syncwarp();
+            if (lane == 0) {
+                if (2 * sw < nc) mbar_arrive(smem_u32(&sm.empty[it.stage(2 * sw)]));          // the producer may refill them
+                if (2 * sw + 1 < nc) mbar_arrive(smem_u32(&sm.empty[it.stage(2 * sw + 1)]));
+                mbar_arrive(smem_u32(&sm.passb_done[slot]));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ ranking
+#pragma unroll 1
+        for (ItemIter it(p, (int)sizeof(T)); it.valid(); it.next()) {
+            const uint32_t slot = it.slot();
+            if (!mbar_wait_warp(smem_u32(&sm.passb_done[slot]), it.slot_phase(), abort_flag)) break;
+            const int n = sm.cand_count[slot];
+            const int64_t out = (int64_t)it.row() * p.S + it.seg();
             float* tv = p.top_val + out * p.K1;
             int32_t* ti = p.top_idx + out * p.K1;
             if (n <= kCandCap) {
-                // release the stages first, the ordering below only needs the candidate list
-                if (lane == 0)
-                    for (int c2 = 0; c2 < n_chunks; ++c2) mbar_arrive(smem_u32(&sm.empty[(fills_end - n_chunks + c2) % kStages]));
-                for (int i = stid; i < p.K1; i += kSelThreads) if (i >= n) { tv[i] = neg_inf(); ti[i] = -1; }
-                for (int i = stid; i < n; i += kSelThreads) {
-                    const uint64_t ki = sm.cand[i];
+#pragma unroll 1
+                for (int i = n + lane; i < p.K1; i += 32) { tv[i] = neg_inf(); ti[i] = -1; }
+#pragma unroll 1
+                for (int i = lane; i < n; i += 32) {
+                    const uint64_t ki = sm.cand[slot][i];
                     int rank = 0;
-                    for (int j = 0; j < n; ++j) rank += sm.cand[j] > ki;
+#pragma unroll 2
+                    for (int j = 0; j < n; ++j) rank += sm.cand[slot][j] > ki;
                     if (rank < p.K1) { tv[rank] = row_key_val(ki); ti[rank] = row_key_idx(ki); }
                 }
             } else {
-                // too many entries at or above the bound (long runs of equal values, or an adversarial
-                // layout): take the K1 best one at a time from the chunks, which are still resident
-                uint64_t prev = ~0ull;
-                for (int r2 = 0; r2 < p.K1; ++r2) {
-                    uint64_t best = 0;
-                    for (int c2 = 0; c2 < n_chunks; ++c2) {
-                        const uint32_t st = (fills_end - n_chunks + c2) % kStages;
-                        const int bytes = min(kChunkBytes, bytes_item - c2 * kChunkBytes);
-                        const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[st]);
-                        for (int vi = stid; vi < (bytes >> 4); vi += kSelThreads) {
-                            float x[kElems];
-                            Vec<T>::unpack(vec[vi], x);
-                            const int base = elem0 + c2 * kChunkElems + vi * kElems;
-#pragma unroll
-                            for (int e = 0; e < kElems; ++e) {
-                                const uint64_t kk = row_key(x[e], base + e);
-                                if (kk < prev && kk > best) best = kk;
-                            }
-                        }
-                    }
-                    best = warp_max_u64(best);
-                    if (lane == 0) sm.red[sw] = best;
-                    sel_barrier();
-                    best = sm.red[0];
-#pragma unroll
-                    for (int w = 1; w < kNS; ++w) best = sm.red[w] > best ? sm.red[w] : best;
-                    sel_barrier();
-                    if (stid == 0) { tv[r2] = best ? row_key_val(best) : neg_inf(); ti[r2] = best ? row_key_idx(best) : -1; }
-                    prev = best;      // 0 once exhausted: nothing is below it
-                }
-                if (lane == 0)
-                    for (int c2 = 0; c2 < n_chunks; ++c2) mbar_arrive(smem_u32(&sm.empty[(fills_end - n_chunks + c2) % kStages]));
+                rank_from_global<T>((const T*)p.logits + (int64_t)it.row() * p.stride, it.seg() * p.seg_len,
+                                    it.seg() * p.seg_len + it.bytes() / (int)sizeof(T), p.K1, tv, ti);
             }
-            sel_barrier();
-            if (stid == 0) sm.cand_count = 0;
-            sel_barrier();
+            __syncwarp();
+            if (lane == 0) { sm.cand_count[slot] = 0; mbar_arrive(smem_u32(&sm.slot_free[slot])); }
         }
     }
     __syncthreads();
