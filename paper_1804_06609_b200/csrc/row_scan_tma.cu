@@ -7,12 +7,13 @@
 //   consumers   each warp streams half a chunk of the item: the maximum first, then exp2(x*log2e - c) summed per
 //               lane (Section 2's normaliser) with c a whole number at or above the maximum; it leaves one
 //               maximum per lane; no selection logic in this loop;
-//   bound       one warp turns the lane maxima into a lower bound of the K1-th largest entry of the item: the
-//               K1-th largest of maxima of disjoint groups is one; found exactly by bisection on ordered keys;
+//   bound       warps (alternating items) turn the lane maxima into a lower bound of the K1-th largest entry of
+//               the item: the K1-th largest of maxima of disjoint groups is one; found by bisection on the
+//               leading 16 bits of an ordered key;
 //   pass B      warps look again only at the vectors of lanes whose maximum reaches the bound (a few dozen of
 //               the 4096 vectors of an item), collect the entries at or above the bound, and hand the stages
 //               back to the producer;
-//   ranking     one warp orders the collected entries exactly (value descending, lower index first) and
+//   ranking     warps (alternating items) order the collected entries exactly (value descending, lower index first) and
 //               writes the segment's partial result.
 // Every wait is bounded: a wait that runs out sets the timeout bit of the status word and the CTA winds down.
 // The code is kept small on purpose: the roles run different code at the same time and share one
@@ -33,11 +34,13 @@ constexpr int kVecsPerLane = kHalfVecs / 32;   // 8
 constexpr int kStages = 24;                    // 192 KB of ring
 constexpr int kMaxSegChunks = 8;               // a segment is at most 64 KB
 constexpr int kNC = 2 * kMaxSegChunks;         // consumer warps, half a chunk of the item each
-constexpr int kNS = 4;                         // pass-B warps, two chunks of the item each
-constexpr int kWarpBound = 1 + kNC;            // warp index of the bound warp
-constexpr int kWarpPassB = kWarpBound + 1;     // first pass-B warp
-constexpr int kWarpRank = kWarpPassB + kNS;    // ranking warp
-constexpr int kThreads = 32 * (kWarpRank + 1);
+constexpr int kNB = 2;                         // bound warps, alternating items
+constexpr int kNS = kMaxSegChunks;             // pass-B warps, one chunk of the item each
+constexpr int kNR = 2;                         // ranking warps, alternating items
+constexpr int kWarpBound = 1 + kNC;            // first bound warp
+constexpr int kWarpPassB = kWarpBound + kNB;   // first pass-B warp
+constexpr int kWarpRank = kWarpPassB + kNS;    // first ranking warp
+constexpr int kThreads = 32 * (kWarpRank + kNR);
 constexpr int kSlots = 4;                      // items in flight between consumers and ranking
 constexpr int kCandCap = 256;                  // entries at or above the bound that one item may hold
 constexpr uint32_t kSpinLimit = 1u << 20;
@@ -322,68 +325,51 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sm.item_done[it.slot()]));
         }
-    } else if (warp == kWarpBound) {
+    } else if (warp < kWarpPassB) {
         // ------------------------------------------------------------------ bound
+        const int bw = warp - kWarpBound;
 #pragma unroll 1
         for (ItemIter it(p, (int)sizeof(T)); it.valid(); it.next()) {
+            if ((int)(it.n_item % kNB) != bw) continue;       // the other bound warp's item
             const uint32_t slot = it.slot();
             if (!mbar_wait_warp(smem_u32(&sm.item_done[slot]), it.slot_phase(), abort_flag)) break;
-            // K1-th largest of 256 group maxima (a group = the two lanes that share a chunk position), exactly,
-            // by bisection on their ordered keys (bf16 values need 16 key bits, fp32 values 32); the bits all
-            // keys share are skipped
-            constexpr int kKeyBits = sizeof(T) == 2 ? 16 : 32;
+            // The K1-th largest of 256 group maxima (a group = the two lanes that share a chunk position), to
+            // the leading 16 bits of the ordered key (all of a bf16 value; sign, exponent and 7 mantissa bits
+            // of an fp32 one), by bisection two bits at a time; the bits all keys share are skipped.
             constexpr int kGroups = kNC / 2;
             uint32_t key[kGroups], orv = 0, andv = ~0u;
 #pragma unroll
             for (int w = 0; w < kGroups; ++w) {
-                key[w] = ord32(fmaxf(sm.lane_max[slot][2 * w][lane], sm.lane_max[slot][2 * w + 1][lane])) >> (32 - kKeyBits);
+                key[w] = ord32(fmaxf(sm.lane_max[slot][2 * w][lane], sm.lane_max[slot][2 * w + 1][lane])) >> 16;
                 orv |= key[w]; andv &= key[w];
             }
             orv = __reduce_or_sync(kFullMask, orv); andv = __reduce_and_sync(kFullMask, andv);
             uint32_t t = andv;
             if (orv != andv) {
-                const int top = 31 - __clz(orv ^ andv);
+                const int top = (31 - __clz(orv ^ andv)) | 1;          // highest differing bit, rounded up to a pair
                 t = andv & ~((2u << top) - 1u);
 #pragma unroll 1
-                for (int bit = top; bit >= 0; --bit) {
-                    const uint32_t c = t | (1u << bit);
-                    int cnt = 0;
+                for (int bit = top - 1; bit >= 0; bit -= 2) {
+                    const uint32_t c1 = t | (1u << bit), c2 = t | (2u << bit), c3 = t | (3u << bit);
+                    int n1 = 0, n2 = 0, n3 = 0;
 #pragma unroll
-                    for (int w = 0; w < kGroups; ++w) cnt += key[w] >= c;
-                    if ((int)__reduce_add_sync(kFullMask, cnt) >= p.K1) t = c;
+                    for (int w = 0; w < kGroups; ++w) { n1 += key[w] >= c1; n2 += key[w] >= c2; n3 += key[w] >= c3; }
+                    n1 = __reduce_add_sync(kFullMask, n1); n2 = __reduce_add_sync(kFullMask, n2); n3 = __reduce_add_sync(kFullMask, n3);
+                    t = n3 >= p.K1 ? c3 : n2 >= p.K1 ? c2 : n1 >= p.K1 ? c1 : t;
                 }
             }
             if (lane == 0) {
-                uint32_t o = t;
-                if (kKeyBits == 16) o = (t << 16) | ((t & 0x8000u) ? 0u : 0xffffu);   // a bf16 value's low key bits
-                sm.bound_lo[slot] = unord32(o);      // an actual lane maximum (possibly -inf)
-                // the segment's normaliser: sum_x 2^(x*log2e) = S * 2^C with a whole number C
-                float C = neg_inf();
-#pragma unroll 1
-                for (int w = 0; w < kNC; ++w) C = fmaxf(C, sm.warp_ref[slot][w]);
-                float m = neg_inf(), s2 = 0.f;
-                if (C != neg_inf()) {
-                    float S = 0.f;
-#pragma unroll 1
-                    for (int w = 0; w < kNC; ++w) {
-                        const float cw2 = sm.warp_ref[slot][w];
-                        if (cw2 != neg_inf()) S += sm.warp_sum[slot][w] * pow2i((int)(cw2 - C));
-                    }
-                    // (m, s) with sum_x e^x = s * e^m: m = fl32(C ln2), the rounding of m folded into s
-                    constexpr float kLn2Hi = 0.693147182464599609375f, kLn2Lo = -1.904654299957767e-9f;
-                    m = C * kLn2Hi;
-                    const float err = fmaf(C, kLn2Hi, -m) + C * kLn2Lo;
-                    s2 = fmaf(S, err, S);
-                }
-                const int64_t out = (int64_t)it.row() * p.S + it.seg();
-                p.part_m[out] = m; p.part_s[out] = s2;
+                // the smallest value with these leading key bits: at least K1 entries of the item reach it
+                float lo = unord32(t << 16);
+                if (!(lo == lo)) lo = neg_inf();          // the bucket that holds -inf has no finite lower edge
+                sm.bound_lo[slot] = lo;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sm.bound_ready[slot]));
         }
     } else if (warp < kWarpRank) {
         // ------------------------------------------------------------------ pass B
-        // This warp owns consumer warps 4*sw .. 4*sw+3, i.e. chunks 2*sw and 2*sw+1 of every item.  Only lanes
+        // This warp owns chunk sw of every item, i.e. consumer warps 2*sw and 2*sw+1.  Only lanes
         // whose maximum reaches the bound can hold an entry at or above it; up to four such lanes are handled
         // at a time, eight lanes of this warp looking at the eight vectors of one of them.
         const int sw = warp - kWarpPassB, grp = lane >> 3, vrow = lane & 7;
@@ -397,8 +383,8 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
             const int nc = it.n_chunks();
             const int elem0 = it.seg() * p.seg_len;
 #pragma unroll 1
-            for (int q = 0; q < 4; ++q) {
-                const int w = 4 * sw + q, chunk = w >> 1, half = w & 1;
+            for (int q = 0; q < 2; ++q) {
+                const int w = 2 * sw + q, chunk = sw, half = q;
                 if (chunk >= nc) break;
                 unsigned m = __ballot_sync(kFullMask, sm.lane_max[slot][w][lane] >= lo);
                 const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[it.stage(chunk)]);
@@ -425,8 +411,7 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
             }
             __syncwarp();
             if (lane == 0) {
-                if (2 * sw < nc) mbar_arrive(smem_u32(&sm.empty[it.stage(2 * sw)]));          // the producer may refill them
-                if (2 * sw + 1 < nc) mbar_arrive(smem_u32(&sm.empty[it.stage(2 * sw + 1)]));
+                if (sw < nc) mbar_arrive(smem_u32(&sm.empty[it.stage(sw)]));          // the producer may refill it
                 mbar_arrive(smem_u32(&sm.passb_done[slot]));
             }
         }
@@ -434,10 +419,27 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
         // ------------------------------------------------------------------ ranking
 #pragma unroll 1
         for (ItemIter it(p, (int)sizeof(T)); it.valid(); it.next()) {
+            if ((int)(it.n_item % kNR) != warp - kWarpRank) continue;       // the other ranking warp's item
             const uint32_t slot = it.slot();
             if (!mbar_wait_warp(smem_u32(&sm.passb_done[slot]), it.slot_phase(), abort_flag)) break;
             const int n = sm.cand_count[slot];
             const int64_t out = (int64_t)it.row() * p.S + it.seg();
+            {   // the segment's normaliser: sum_x 2^(x*log2e) = S * 2^C with a whole number C; lane w holds warp w's part
+                const float cw2 = lane < kNC ? sm.warp_ref[slot][lane] : neg_inf();
+                const float C = warp_max(cw2);
+                const float S = warp_sum(cw2 != neg_inf() ? sm.warp_sum[slot][lane] * pow2i((int)(cw2 - C)) : 0.f);
+                if (lane == 0) {
+                    float m = neg_inf(), s2 = 0.f;
+                    if (C != neg_inf()) {
+                        // (m, s) with sum_x e^x = s * e^m: m = fl32(C ln2), the rounding of m folded into s
+                        constexpr float kLn2Hi = 0.693147182464599609375f, kLn2Lo = -1.904654299957767e-9f;
+                        m = C * kLn2Hi;
+                        const float err = fmaf(C, kLn2Hi, -m) + C * kLn2Lo;
+                        s2 = fmaf(S, err, S);
+                    }
+                    p.part_m[out] = m; p.part_s[out] = s2;
+                }
+            }
             float* tv = p.top_val + out * p.K1;
             int32_t* ti = p.top_idx + out * p.K1;
             if (n <= kCandCap) {
