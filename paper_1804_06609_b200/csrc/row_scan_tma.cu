@@ -7,9 +7,9 @@
 //   consumers   each warp streams half a chunk of the item: the maximum first, then exp2(x*log2e - c) summed per
 //               lane (Section 2's normaliser) with c a whole number at or above the maximum; it leaves one
 //               maximum per lane; no selection logic in this loop;
-//   bound       warps (alternating items) turn the lane maxima into a lower bound of the K1-th largest entry of
-//               the item: the K1-th largest of maxima of disjoint groups is one; found by bisection on the
-//               leading 16 bits of an ordered key;
+//   bound       every consumer warp also leaves its J largest lane maxima; a warp takes the K1-th largest of
+//               these values as a lower bound of the K1-th largest entry of the item (maxima of disjoint lanes:
+//               at least K1 entries reach it).  J = ceil(K1 / warps with data), 2 for the usual shapes;
 //   pass B      warps look again only at the vectors of lanes whose maximum reaches the bound (a few dozen of
 //               the 4096 vectors of an item), collect the entries at or above the bound, and hand the stages
 //               back to the producer;
@@ -34,7 +34,7 @@ constexpr int kVecsPerLane = kHalfVecs / 32;   // 8
 constexpr int kStages = 24;                    // 192 KB of ring
 constexpr int kMaxSegChunks = 8;               // a segment is at most 64 KB
 constexpr int kNC = 2 * kMaxSegChunks;         // consumer warps, half a chunk of the item each
-constexpr int kNB = 2;                         // bound warps, alternating items
+constexpr int kNB = 1;                         // bound warps
 constexpr int kNS = kMaxSegChunks;             // pass-B warps, one chunk of the item each
 constexpr int kNR = 2;                         // ranking warps, alternating items
 constexpr int kWarpBound = 1 + kNC;            // first bound warp
@@ -57,6 +57,7 @@ struct Smem {
     uint64_t slot_free[kSlots];
     uint64_t cand[kSlots][kCandCap];
     float lane_max[kSlots][kNC][32];
+    float lane_top[kSlots][kNC * 32];       // the J largest lane maxima of consumer warp w at [w*J, w*J + J)
     float warp_sum[kSlots][kNC];
     float warp_ref[kSlots][kNC];            // the whole number c of exp2(x*log2e - c) each warp used (-inf: no data)
     float bound_lo[kSlots];                 // entries >= bound_lo are collected
@@ -209,6 +210,10 @@ struct ItemIter {
     __device__ uint32_t stage(int c) const { return (fills + (uint32_t)c) % kStages; }
     __device__ uint32_t stage_phase(int c) const { return ((fills + (uint32_t)c) / kStages) & 1u; }
     __device__ int chunk_vecs(int c) const { return min(kChunkBytes, bytes_ - c * kChunkBytes) >> 4; }
+    // consumer warps that get data (half a chunk each), and how many lane maxima each reports so that
+    // together they report at least K1 (capped by the 32 lanes a warp has)
+    __device__ int active_warps() const { return ((bytes_ >> 4) + kHalfVecs - 1) / kHalfVecs; }
+    __device__ int report(int K1) const { return min(32, (K1 + active_warps() - 1) / active_warps()); }
 };
 
 // Ranking, rare path: more entries at or above the bound than the list holds (long runs of equal values at the
@@ -320,6 +325,17 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
             // hand the lane maxima and the warp's sum over
             if (!mbar_wait_warp(smem_u32(&sm.slot_free[it.slot()]), it.slot_phase() ^ 1u, abort_flag)) break;
             sm.lane_max[it.slot()][cw][lane] = lmax;
+            if (nvec > 0) {       // the warp's J largest lane maxima, one lane removed per round
+                const int J = it.report(p.K1);
+                float cur = lmax;
+#pragma unroll 1
+                for (int j = 0; j < J; ++j) {
+                    const float m = warp_max(cur);
+                    const unsigned who = __ballot_sync(kFullMask, cur == m);
+                    if (lane == 0) sm.lane_top[it.slot()][cw * J + j] = m;
+                    if (lane == __ffs(who) - 1) cur = neg_inf();
+                }
+            }
             const float wsum = warp_sum(ssum);
             if (lane == 0) { sm.warp_sum[it.slot()][cw] = wsum; sm.warp_ref[it.slot()][cw] = cref; }
             __syncwarp();
@@ -327,43 +343,30 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
         }
     } else if (warp < kWarpPassB) {
         // ------------------------------------------------------------------ bound
-        const int bw = warp - kWarpBound;
 #pragma unroll 1
         for (ItemIter it(p, (int)sizeof(T)); it.valid(); it.next()) {
-            if ((int)(it.n_item % kNB) != bw) continue;       // the other bound warp's item
             const uint32_t slot = it.slot();
             if (!mbar_wait_warp(smem_u32(&sm.item_done[slot]), it.slot_phase(), abort_flag)) break;
-            // The K1-th largest of 256 group maxima (a group = the two lanes that share a chunk position), to
-            // the leading 16 bits of the ordered key (all of a bf16 value; sign, exponent and 7 mantissa bits
-            // of an fp32 one), by bisection two bits at a time; the bits all keys share are skipped.
-            constexpr int kGroups = kNC / 2;
-            uint32_t key[kGroups], orv = 0, andv = ~0u;
-#pragma unroll
-            for (int w = 0; w < kGroups; ++w) {
-                key[w] = ord32(fmaxf(sm.lane_max[slot][2 * w][lane], sm.lane_max[slot][2 * w + 1][lane])) >> 16;
-                orv |= key[w]; andv &= key[w];
-            }
-            orv = __reduce_or_sync(kFullMask, orv); andv = __reduce_and_sync(kFullMask, andv);
-            uint32_t t = andv;
-            if (orv != andv) {
-                const int top = (31 - __clz(orv ^ andv)) | 1;          // highest differing bit, rounded up to a pair
-                t = andv & ~((2u << top) - 1u);
+            // The K1-th largest of the reported lane maxima, by counting for each value how many are larger
+            // (equal values ordered by position, so that the ranks are all different).
+            const int J = it.report(p.K1), T = it.active_warps() * J;
+            float lo = neg_inf();                 // fewer than K1 values: everything is collected
+            if (T >= p.K1) {
 #pragma unroll 1
-                for (int bit = top - 1; bit >= 0; bit -= 2) {
-                    const uint32_t c1 = t | (1u << bit), c2 = t | (2u << bit), c3 = t | (3u << bit);
-                    int n1 = 0, n2 = 0, n3 = 0;
-#pragma unroll
-                    for (int w = 0; w < kGroups; ++w) { n1 += key[w] >= c1; n2 += key[w] >= c2; n3 += key[w] >= c3; }
-                    n1 = __reduce_add_sync(kFullMask, n1); n2 = __reduce_add_sync(kFullMask, n2); n3 = __reduce_add_sync(kFullMask, n3);
-                    t = n3 >= p.K1 ? c3 : n2 >= p.K1 ? c2 : n1 >= p.K1 ? c1 : t;
+                for (int i0 = 0; i0 < T; i0 += 32) {
+                    const int i = i0 + lane;
+                    const float mine = i < T ? sm.lane_top[slot][i] : neg_inf();
+                    int rank = 0;
+#pragma unroll 4
+                    for (int j = 0; j < T; ++j) {
+                        const float o = sm.lane_top[slot][j];
+                        rank += (o > mine) || (o == mine && j < i);
+                    }
+                    const unsigned hit = __ballot_sync(kFullMask, i < T && rank == p.K1 - 1);
+                    if (hit) lo = __shfl_sync(kFullMask, mine, __ffs(hit) - 1);
                 }
             }
-            if (lane == 0) {
-                // the smallest value with these leading key bits: at least K1 entries of the item reach it
-                float lo = unord32(t << 16);
-                if (!(lo == lo)) lo = neg_inf();          // the bucket that holds -inf has no finite lower edge
-                sm.bound_lo[slot] = lo;
-            }
+            if (lane == 0) sm.bound_lo[slot] = lo;
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sm.bound_ready[slot]));
         }
@@ -382,22 +385,25 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
             const float lo = sm.bound_lo[slot];
             const int nc = it.n_chunks();
             const int elem0 = it.seg() * p.seg_len;
-#pragma unroll 1
-            for (int q = 0; q < 2; ++q) {
-                const int w = 2 * sw + q, chunk = sw, half = q;
-                if (chunk >= nc) break;
-                unsigned m = __ballot_sync(kFullMask, sm.lane_max[slot][w][lane] >= lo);
-                const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[it.stage(chunk)]);
-                const int nvec = it.chunk_vecs(chunk);
-                while (m) {
-                    unsigned mm = m;                                   // the grp-th lowest set bit, if there is one
-                    for (int j = 0; j < grp; ++j) mm &= mm - 1;
+            if (sw < nc) {
+                // bit l of m0 / m1: lane l of the first / second half's consumer warp reaches the bound
+                unsigned m0 = __ballot_sync(kFullMask, sm.lane_max[slot][2 * sw][lane] >= lo);
+                unsigned m1 = __ballot_sync(kFullMask, sm.lane_max[slot][2 * sw + 1][lane] >= lo);
+                const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[it.stage(sw)]);
+                const int nvec = it.chunk_vecs(sw);
+                while (m0 | m1) {
+                    // the grp-th of the remaining candidate lanes, first half before second
+                    int half = 0; unsigned mm = m0;
+                    int skip = grp;
+                    const int c0 = __popc(m0);
+                    if (skip >= c0) { half = 1; mm = m1; skip -= c0; }
+                    for (int j = 0; j < skip; ++j) mm &= mm - 1;
                     const int src_lane = __ffs(mm) - 1;
                     const int vi = half * kHalfVecs + vrow * 32 + src_lane;
                     if (mm && vi < nvec) {
                         float x[kElems];
                         Vec<T>::unpack(vec[vi], x);
-                        const int base = elem0 + chunk * kChunkElems + vi * kElems;
+                        const int base = elem0 + sw * kChunkElems + vi * kElems;
 #pragma unroll
                         for (int e = 0; e < kElems; ++e)
                             if (x[e] >= lo) {
@@ -405,7 +411,8 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
                                 if (pos < kCandCap) sm.cand[slot][pos] = row_key(x[e], base + e);
                             }
                     }
-                    m &= m - 1; m &= m - 1; m &= m - 1; m &= m - 1;     // four lanes done
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) { if (m0) m0 &= m0 - 1; else m1 &= m1 - 1; }     // four lanes done
                     __syncwarp();
                 }
             }
