@@ -34,6 +34,8 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="serving")
     ap.add_argument("--C", type=int, default=None, help="constraint count of the 'scaling' workload")
+    ap.add_argument("--B", type=int, default=None, help="fewer sentences than the workload has (for profiling a small case)")
+    ap.add_argument("--stream-steps", type=int, default=None, help="keep only the first steps of the stream resident")
     ap.add_argument("--e2e-steps", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -46,12 +48,20 @@ def measured_peak():
     return 6650.0, "fallback"
 
 
-def ncu_traffic(workload):
-    """DRAM bytes per row-scan launch from the last ncu capture, if the kernel has not changed since."""
-    p = os.path.join(ROOT, "profiles", "row_scan_traffic.json")
-    if os.path.exists(p):
-        d = json.load(open(p))
-        return d.get(workload)
+def ncu_traffic(workload, open_rows_per_launch):
+    """DRAM bytes (read + write) per row-scan launch, scaled from the committed ncu capture of a smaller case
+    by the rows a launch processes (traffic grows in proportion: one pass per open row).  None when the
+    kernel source has changed since the counters were taken."""
+    import hashlib
+    p = os.path.join(ROOT, "profiles", "row_scan_traffic.txt")
+    src = os.path.join(ROOT, "paper_1804_06609_b200", "csrc", "row_scan_tma.cu")
+    if not (os.path.exists(p) and os.path.exists(src)):
+        return None
+    digest = hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+    for line in open(p):
+        f = line.split()
+        if len(f) == 3 and f[0] == workload and f[1] == digest:
+            return float(f[2]) * open_rows_per_launch
     return None
 
 
@@ -90,7 +100,8 @@ class ClockSampler(threading.Thread):
 
 def workload_of(args):
     from synth_inputs import make_workload
-    return make_workload(args.workload, C=args.C)
+    kw = {"B": args.B} if args.B else {}
+    return make_workload(args.workload, C=args.C, **kw)
 
 
 # ---------------------------------------------------------------------------------------------- oracle
@@ -165,7 +176,7 @@ def run_ours(args):
     esize = 2 if wl.dtype == "bf16" else 4
     step_bytes = wl.R * wl.V * esize
     free, _ = torch.cuda.mem_get_info(dev)
-    T = int(max(1, min(wl.steps, (free * 0.6) // step_bytes)))
+    T = int(max(1, min(wl.steps, (free * 0.6) // step_bytes, args.stream_steps or wl.steps)))
     # rotate enough distinct step buffers that consecutive steps never find their input in L2
     gen = GpuLogitStream(wl, dev)
     st = pkg.DbaStepper(wl.B, wl.k, wl.V, wl.steps, constraints=wl.constraints,
@@ -230,7 +241,7 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     scan_ms = kt[0] / ksteps
     achieved = kbytes / ksteps / (scan_ms / 1e3) / 1e9
-    traffic = ncu_traffic(wl.name)
+    traffic = ncu_traffic(wl.name, kbytes / ksteps / (wl.V * esize))
 
     # --- end to end: host logits in pinned memory, outputs read back, through dba_step_host ------------
     Th = min(T, 8)
