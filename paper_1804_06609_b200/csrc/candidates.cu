@@ -10,7 +10,7 @@ namespace dba {
 
 namespace {
 
-constexpr int kCandThreads = 256;
+constexpr int kCandThreads = 512;
 constexpr int kCandWarps = kCandThreads / 32;
 
 struct SortEnt {
@@ -286,27 +286,34 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
 
     // ---- phase B (source 1): the k best cells of the whole matrix, by a k-round tournament of row heads ----
     if (warp == 0) {
+        // lane l holds the heads of rows l and l + 32: ordered score key and flat index of the best unused cell
+        uint32_t ks[2]; int fl[2], ptr[2] = {0, 0};
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int h = lane + 32 * q;
+            const bool has = h < k && rt_n[h] > 0;
+            ks[q] = has ? ord32(rt_score[h * k]) : 0u;            // 0 is below every real key
+            fl[q] = has ? h * V + rt_w[h * k] : 0x7fffffff;
+        }
         int ns1 = 0;
         for (int round = 0; round < k; ++round) {
-            float bs = neg_inf(); int bf = 0x7fffffff; int bh = -1;
-            for (int h = lane; h < k; h += 32) {
-                const int p = rt_ptr[h];
-                if (p < rt_n[h]) {
-                    const float s = rt_score[h * k + p]; const int f = h * V + rt_w[h * k + p];
-                    if (bh < 0 || cell_better(s, f, bs, bf)) { bs = s; bf = f; bh = h; }
-                }
+            // best head: highest score key, then lowest flat index
+            const int q = (ks[1] > ks[0] || (ks[1] == ks[0] && fl[1] < fl[0])) ? 1 : 0;
+            const uint32_t kmax = __reduce_max_sync(kFullMask, q ? ks[1] : ks[0]);
+            if (kmax == 0u) break;
+            const int mine = (q ? ks[1] : ks[0]) == kmax ? (q ? fl[1] : fl[0]) : 0x7fffffff;
+            const int fmin = __reduce_min_sync(kFullMask, mine);
+            if (mine == fmin) {                                    // exactly one lane: flat indices are distinct
+                const int h = lane + 32 * q;
+                s1_h[ns1] = h; s1_i[ns1] = q ? ptr[1] : ptr[0];
+                const int np = (q ? ptr[1] : ptr[0]) + 1;
+                const bool has = np < rt_n[h];
+                const uint32_t nk = has ? ord32(rt_score[h * k + np]) : 0u;
+                const int nf = has ? h * V + rt_w[h * k + np] : 0x7fffffff;
+                if (q) { ptr[1] = np; ks[1] = nk; fl[1] = nf; } else { ptr[0] = np; ks[0] = nk; fl[0] = nf; }
+                rt_ptr[h] = np;
             }
-#pragma unroll
-            for (int o = 16; o; o >>= 1) {
-                const float os = __shfl_xor_sync(kFullMask, bs, o);
-                const int of = __shfl_xor_sync(kFullMask, bf, o);
-                const int oh = __shfl_xor_sync(kFullMask, bh, o);
-                if (oh >= 0 && (bh < 0 || cell_better(os, of, bs, bf))) { bs = os; bf = of; bh = oh; }
-            }
-            if (bh < 0) break;
-            if (lane == 0) { s1_h[ns1] = bh; s1_i[ns1] = rt_ptr[bh]; rt_ptr[bh] += 1; }
             ++ns1;
-            __syncwarp();
         }
         if (lane == 0) s_ns1 = ns1;
     }
@@ -361,7 +368,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     int n = s_ncand;
     if (n > d.max_cand) { if (tid == 0) atomicOr(status, kStatusOverflow); n = d.max_cand; }
 
-    // ---- group by bank, order inside each bank (Section 3.1): bitonic sort on (bank, score desc, flat asc) --
+    // ---- group by bank, order inside each bank (Section 3.1): order (bank asc, score desc, flat asc) ---------
     int n_sort = 32;
     while (n_sort < n) n_sort <<= 1;
     for (int i = tid; i < n_sort; i += kCandThreads) {
@@ -373,22 +380,36 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         ent[i] = e;
     }
     __syncthreads();
-    for (int size = 2; size <= n_sort; size <<= 1) {
-        for (int str = size >> 1; str > 0; str >>= 1) {
-            for (int t = tid; t < n_sort / 2; t += kCandThreads) {
-                const int pos = 2 * t - (t & (str - 1));
-                SortEnt a = ent[pos], c = ent[pos + str];
-                const bool gt = a.hi > c.hi || (a.hi == c.hi && a.lo > c.lo);
-                const bool up = (pos & size) == 0;
-                if (gt == up) { ent[pos] = c; ent[pos + str] = a; }
+    if (n <= kCandThreads) {
+        // short list: every thread counts how many entries precede its own (keys are distinct) and writes it there
+        if (tid < n) {
+            const SortEnt me = ent[tid];
+            int rank = 0;
+            for (int j = 0; j < n; ++j) {
+                const SortEnt o = ent[j];
+                rank += o.hi < me.hi || (o.hi == me.hi && o.lo < me.lo);
             }
-            __syncthreads();
+            Cand c; c.score = c_score[tid]; c.flat = c_flat[tid]; c.mask = c_mask[tid]; c.active = c_active[tid]; c.pad_ = 0;
+            cand_out[(int64_t)b * d.max_cand + rank] = c;
         }
-    }
-    for (int i = tid; i < n; i += kCandThreads) {
-        const int id = ent[i].id;
-        Cand c; c.score = c_score[id]; c.flat = c_flat[id]; c.mask = c_mask[id]; c.active = c_active[id]; c.pad_ = 0;
-        cand_out[(int64_t)b * d.max_cand + i] = c;
+    } else {
+        for (int size = 2; size <= n_sort; size <<= 1) {
+            for (int str = size >> 1; str > 0; str >>= 1) {
+                for (int t = tid; t < n_sort / 2; t += kCandThreads) {
+                    const int pos = 2 * t - (t & (str - 1));
+                    SortEnt a = ent[pos], c = ent[pos + str];
+                    const bool gt = a.hi > c.hi || (a.hi == c.hi && a.lo > c.lo);
+                    const bool up = (pos & size) == 0;
+                    if (gt == up) { ent[pos] = c; ent[pos + str] = a; }
+                }
+                __syncthreads();
+            }
+        }
+        for (int i = tid; i < n; i += kCandThreads) {
+            const int id = ent[i].id;
+            Cand c; c.score = c_score[id]; c.flat = c_flat[id]; c.mask = c_mask[id]; c.active = c_active[id]; c.pad_ = 0;
+            cand_out[(int64_t)b * d.max_cand + i] = c;
+        }
     }
     if (tid <= kMaxC) bank_count[b * (kMaxC + 1) + tid] = bank_cnt[tid];
     if (tid == 0) ncand_out[b] = n;
