@@ -163,17 +163,13 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
             if (lane == 0) { rt_n[h] = 1; rt_score[h * k] = s_parent[h]; rt_w[h * k] = d.eos_id; row_lse[r] = 0.f; s_lse[h] = 0.f; }
             continue;
         }
-        // row normaliser from the segment partials (fixed order)
+        // row normaliser from the segment partials: lane g holds segment g (S <= 8), fixed reduction order
         float lse;
         {
-            float M = neg_inf();
-            for (int g = 0; g < S; ++g) M = fmaxf(M, part.m[r * S + g]);
-            float sum = 0.f;
-            if (M != neg_inf())
-                for (int g = 0; g < S; ++g) {
-                    const float mg = part.m[r * S + g];
-                    if (mg != neg_inf()) sum += part.s[r * S + g] * expf(mg - M);
-                }
+            const float mg = lane < S ? part.m[r * S + lane] : neg_inf();
+            const float M = warp_max(mg);
+            const float term = mg != neg_inf() ? part.s[r * S + lane] * expf(mg - M) : 0.f;
+            const float sum = warp_sum(term);
             lse = M == neg_inf() ? neg_inf() : M + logf(sum);
         }
         if (lane == 0) row_lse[r] = lse;
@@ -196,11 +192,21 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
                 stage[e] = ix >= 0 ? row_key(part.top_val[(int64_t)r * n + e], ix) : 0ull;
             }
             __syncwarp();
+            // every segment's list is in descending key order (empty entries, key 0, last): the place of an
+            // entry in the merged order is its place in its own list plus, for every other list, the number of
+            // keys above it, found by bisection
             for (int e = lane; e < n; e += 32) {
                 const uint64_t key = stage[e];
                 if (!key) continue;
-                int rank = 0;
-                for (int j = 0; j < n; ++j) rank += stage[j] > key;
+                const int g = e / K1;
+                int rank = e - g * K1;
+                for (int g2 = 0; g2 < S; ++g2) {
+                    if (g2 == g) continue;
+                    const uint64_t* lst = stage + g2 * K1;
+                    int lo2 = 0, hi2 = K1;                      // first position whose key is not above `key`
+                    while (lo2 < hi2) { const int mid = (lo2 + hi2) >> 1; if (lst[mid] > key) lo2 = mid + 1; else hi2 = mid; }
+                    rank += lo2;
+                }
                 if (rank < K1) merged[rank] = key;
             }
         }
@@ -273,6 +279,14 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         }
         // order by (score desc, token asc), keep the first k and publish
         const int nrow = min(m, k);
+        bool ordered = m <= 32;                               // common case: already in (score desc, token asc) order
+        if (ordered) {
+            const bool bad = lane + 1 < m && !cell_better(tmp_score[lane], tmp_w[lane], tmp_score[lane + 1], tmp_w[lane + 1]);
+            ordered = !__any_sync(kFullMask, bad);
+        }
+        if (ordered) {
+            if (lane < nrow) { rt_score[h * k + lane] = tmp_score[lane]; rt_w[h * k + lane] = tmp_w[lane]; }
+        } else
         for (int i = lane; i < m; i += 32) {
             const float si = tmp_score[i]; const int wi = tmp_w[i];
             int rank = 0;
@@ -316,6 +330,62 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
             ++ns1;
         }
         if (lane == 0) s_ns1 = ns1;
+    } else {
+        // ---- source 2, meanwhile, on the other warps (a row per warp): for every open hypothesis the tokens that
+        //      raise its met count by one.  They all land in the same bank, so of one row at most k can ever be
+        //      kept: with more, only the row's k best go on (the rest could not be selected; the bank still
+        //      counts at least k candidates, which is all the allocation needs to know).
+        for (int h = warp - 1; h < k; h += kCandWarps - 1) {
+            if (s_kind[h] != 1) continue;
+            const uint64_t m = s_mask[h]; const int a = s_active[h];
+            const float lse = s_lse[h], parent = s_parent[h];
+            float sc2[2]; int w2[2], j2[2]; bool v2[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int j = lane + 32 * q;
+                bool ok = j < C && lse != neg_inf();
+                if (ok) {
+                    if (a >= 0) ok = j == a + 1;
+                    else {
+                        ok = ((sc.first_mask >> j) & 1ull) && !((m >> j) & 1ull);
+                        uint64_t earlier = ok ? sc.first_mask & ~m & ((1ull << j) - 1ull) : 0ull;   // same token earlier?
+                        while (earlier) { const int e = __ffsll((long long)earlier) - 1; ok = ok && sc.ctok[e] != sc.ctok[j]; earlier &= earlier - 1; }
+                    }
+                }
+                float x = neg_inf();
+                if (ok) { w2[q] = sc.ctok[j]; x = load_logit_dyn(logits, d.dtype, (int64_t)(r0 + h) * stride + w2[q]); }
+                else w2[q] = 0x7fffffff;
+                v2[q] = ok && x != neg_inf();
+                sc2[q] = v2[q] ? cell_score(x, lse, parent) : neg_inf();
+                j2[q] = j;
+            }
+            const unsigned b0 = __ballot_sync(kFullMask, v2[0]), b1 = __ballot_sync(kFullMask, v2[1]);
+            int cnt = __popc(b0) + __popc(b1);
+            if (cnt > k) {                                    // keep the row's k best (score desc, token asc)
+                int rank[2] = {0, 0};
+                for (int o = 0; o < 32; ++o)
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        const float os = __shfl_sync(kFullMask, sc2[q], o); const int ow = __shfl_sync(kFullMask, w2[q], o);
+                        rank[0] += cell_better(os, ow, sc2[0], w2[0]); rank[1] += cell_better(os, ow, sc2[1], w2[1]);
+                    }
+                v2[0] = v2[0] && rank[0] < k; v2[1] = v2[1] && rank[1] < k;
+                cnt = k;
+            }
+            const unsigned k0 = __ballot_sync(kFullMask, v2[0]), k1 = __ballot_sync(kFullMask, v2[1]);
+            int base = 0;
+            if (lane == 0 && cnt) { base = atomicAdd(&s_ncand, cnt); atomicAdd(&bank_cnt[__popcll(m) + 1], cnt); }
+            base = __shfl_sync(kFullMask, base, 0);
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int slot = base + (q ? __popc(k0) : 0) + __popc((q ? k1 : k0) & lt_mask);
+                if (v2[q] && slot < d.max_cand) {
+                    const int j = j2[q];
+                    c_score[slot] = sc2[q]; c_flat[slot] = h * V + w2[q]; c_mask[slot] = m | (1ull << j);
+                    c_active[slot] = ((sc.last_mask >> j) & 1ull) ? -1 : j;
+                }
+            }
+        }
     }
     __syncthreads();
 
@@ -337,31 +407,6 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         if (slot < d.max_cand) {
             c_score[slot] = rt_score[h * k + i]; c_flat[slot] = h * V + w; c_mask[slot] = m; c_active[slot] = a;
             atomicAdd(&bank_cnt[__popcll(m)], 1);
-        }
-    }
-    // ---- source 2: for every open hypothesis the tokens that raise its met count by one -------------------
-    for (int t = tid; t < k * kMaxC; t += kCandThreads) {
-        const int h = t >> 6, j = t & 63;
-        if (j >= C || s_kind[h] != 1) continue;
-        const uint64_t m = s_mask[h]; const int a = s_active[h];
-        if (a >= 0) { if (j != a + 1) continue; }
-        else {
-            if (!((sc.first_mask >> j) & 1ull) || ((m >> j) & 1ull)) continue;
-            bool dup = false;                              // same token opens an earlier unmet phrase
-            uint64_t earlier = sc.first_mask & ~m & ((1ull << j) - 1ull);
-            while (earlier) { const int q = __ffsll((long long)earlier) - 1; dup |= sc.ctok[q] == sc.ctok[j]; earlier &= earlier - 1; }
-            if (dup) continue;
-        }
-        const int w = sc.ctok[j];
-        const float x = load_logit_dyn(logits, d.dtype, (int64_t)(r0 + h) * stride + w);
-        const float lse = s_lse[h];
-        if (x == neg_inf() || lse == neg_inf()) continue;
-        const int slot = atomicAdd(&s_ncand, 1);
-        if (slot < d.max_cand) {
-            const uint64_t m2 = m | (1ull << j);
-            c_score[slot] = cell_score(x, lse, s_parent[h]); c_flat[slot] = h * V + w; c_mask[slot] = m2;
-            c_active[slot] = ((sc.last_mask >> j) & 1ull) ? -1 : j;
-            atomicAdd(&bank_cnt[__popcll(m2)], 1);
         }
     }
     __syncthreads();

@@ -349,20 +349,20 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
             if (!mbar_wait_warp(smem_u32(&sm.item_done[slot]), it.slot_phase(), abort_flag)) break;
             // The K1-th largest of the reported lane maxima, by counting for each value how many are larger
             // (equal values ordered by position, so that the ranks are all different).
-            const int J = it.report(p.K1), T = it.active_warps() * J;
+            const int J = it.report(p.K1), n_top = it.active_warps() * J;
             float lo = neg_inf();                 // fewer than K1 values: everything is collected
-            if (T >= p.K1) {
+            if (n_top >= p.K1) {
 #pragma unroll 1
-                for (int i0 = 0; i0 < T; i0 += 32) {
+                for (int i0 = 0; i0 < n_top; i0 += 32) {
                     const int i = i0 + lane;
-                    const float mine = i < T ? sm.lane_top[slot][i] : neg_inf();
+                    const float mine = i < n_top ? sm.lane_top[slot][i] : neg_inf();
                     int rank = 0;
 #pragma unroll 4
-                    for (int j = 0; j < T; ++j) {
+                    for (int j = 0; j < n_top; ++j) {
                         const float o = sm.lane_top[slot][j];
                         rank += (o > mine) || (o == mine && j < i);
                     }
-                    const unsigned hit = __ballot_sync(kFullMask, i < T && rank == p.K1 - 1);
+                    const unsigned hit = __ballot_sync(kFullMask, i < n_top && rank == p.K1 - 1);
                     if (hit) lo = __shfl_sync(kFullMask, mine, __ffs(hit) - 1);
                 }
             }
