@@ -10,8 +10,7 @@ namespace dba {
 
 namespace {
 
-constexpr int kCandThreads = 512;
-constexpr int kCandWarps = kCandThreads / 32;
+constexpr int kCandMaxThreads = 1024;      // the host picks 1024, 512 or 256 threads: the most whose scratch fits
 
 struct SortEnt {
     uint64_t hi;   // bank << 32 | (~ordered score): ascending = bank ascending, score descending
@@ -28,7 +27,7 @@ struct Layout {   // byte offsets into dynamic shared memory
 __host__ __device__ inline int align_up(int x, int a) { return (x + a - 1) / a * a; }
 __host__ __device__ inline int next_pow2(int x) { int p = 32; while (p < x) p <<= 1; return p; }
 
-__host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand) {
+__host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand, int n_warps) {
     Layout L;
     int o = 0;
     L.cons = o;      o = align_up(o + (int)sizeof(SentCons), 16);
@@ -45,11 +44,11 @@ __host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand
     L.s1_h = o;      o += 4 * k;
     L.s1_i = o;      o += 4 * k;
     o = align_up(o, 8);
-    L.stage = o;     o += 8 * kCandWarps * (S > 1 ? S * K1 : 0);
-    L.merged = o;    o += 8 * kCandWarps * K1;
-    L.tmp_score = o; o += 4 * kCandWarps * K1;
-    L.tmp_w = o;     o += 4 * kCandWarps * K1;
-    L.tmp_x = o;     o += 4 * kCandWarps * K1;
+    L.stage = o;     o += 8 * n_warps * (S > 1 ? S * K1 : 0);
+    L.merged = o;    o += 8 * n_warps * K1;
+    L.tmp_score = o; o += 4 * n_warps * K1;
+    L.tmp_w = o;     o += 4 * n_warps * K1;
+    L.tmp_x = o;     o += 4 * n_warps * K1;
     o = align_up(o, 8);
     L.c_mask = o;    o += 8 * max_cand;
     L.c_score = o;   o += 4 * max_cand;
@@ -63,41 +62,15 @@ __host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand
     return L;
 }
 
-// constraints[h].add(w): Section 3.1 (last paragraph).  Continue the begun phrase if w is its next token;
-// otherwise reset that phrase's marks and let w open the first wholly unmet word/phrase it matches.
-__device__ __forceinline__ void cons_add(const SentCons& sc, uint64_t& mask, int& active, int w) {
-    if (active >= 0) {
-        const int n = active + 1;
-        if (w == sc.ctok[n]) {
-            mask |= 1ull << n;
-            active = ((sc.last_mask >> n) & 1ull) ? -1 : n;
-            return;
-        }
-        const int p0 = sc.pstart[active];
-        const uint64_t span = ((2ull << active) - 1ull) & ~((1ull << p0) - 1ull);   // bits p0..active
-        mask &= ~span;
-        active = -1;
-    }
-    uint64_t open = sc.first_mask & ~mask;
-    while (open) {
-        const int j = __ffsll((long long)open) - 1;
-        if (sc.ctok[j] == w) {
-            mask |= 1ull << j;
-            active = ((sc.last_mask >> j) & 1ull) ? -1 : j;
-            return;
-        }
-        open &= open - 1;
-    }
-}
-
-__global__ void __launch_bounds__(kCandThreads)
+__global__ void __launch_bounds__(kCandMaxThreads)
 candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const SentCons* __restrict__ cons,
                   Beam cur, ScanOut part, const float* __restrict__ lse_in, float* __restrict__ row_lse,
                   Cand* __restrict__ cand_out, int32_t* __restrict__ ncand_out, int32_t* __restrict__ bank_count,
                   uint32_t* __restrict__ status, int32_t* __restrict__ open_count) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int k = d.k, V = d.V, K1 = d.K1, S = d.S;
-    const Layout L = make_layout(k, K1, S, d.max_cand);
+    const int n_threads = blockDim.x, n_warps = n_threads >> 5;
+    const Layout L = make_layout(k, K1, S, d.max_cand, n_warps);
     SentCons& sc = *reinterpret_cast<SentCons*>(smem + L.cons);
     uint64_t* s_mask = reinterpret_cast<uint64_t*>(smem + L.mask);
     float* s_parent = reinterpret_cast<float*>(smem + L.parent);
@@ -127,7 +100,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     {
         const uint32_t* src = reinterpret_cast<const uint32_t*>(cons + b);
         uint32_t* dst = reinterpret_cast<uint32_t*>(&sc);
-        for (int i = tid; i < (int)(sizeof(SentCons) / 4); i += kCandThreads) dst[i] = src[i];
+        for (int i = tid; i < (int)(sizeof(SentCons) / 4); i += n_threads) dst[i] = src[i];
     }
     if (tid < k) {
         const float ps = cur.score[r0 + tid];
@@ -155,7 +128,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     float* tmp_x = reinterpret_cast<float*>(smem + L.tmp_x) + warp * K1;
     const unsigned lt_mask = (1u << lane) - 1u;
 
-    for (int h = warp; h < k; h += kCandWarps) {
+    for (int h = warp; h < k; h += n_warps) {
         const int r = r0 + h;
         const int kind = s_kind[h];
         if (kind == 0) { if (lane == 0) { row_lse[r] = 0.f; s_lse[h] = 0.f; } continue; }
@@ -163,34 +136,33 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
             if (lane == 0) { rt_n[h] = 1; rt_score[h * k] = s_parent[h]; rt_w[h * k] = d.eos_id; row_lse[r] = 0.f; s_lse[h] = 0.f; }
             continue;
         }
+        // every global load of this row first (they are independent), so that their latencies overlap
+        const int n_ent = S * K1;
+        const float mg = lane < S ? part.m[r * S + lane] : neg_inf();
+        const float sg = lane < S ? part.s[r * S + lane] : 0.f;
+        const float lse_given = lse_in ? lse_in[r] : 0.f;
+        for (int e = lane; e < n_ent; e += 32) {
+            const int ix = part.top_idx[(int64_t)r * n_ent + e];
+            const float xv = part.top_val[(int64_t)r * n_ent + e];
+            (S == 1 ? merged : stage)[e] = ix >= 0 ? row_key(xv, ix) : 0ull;
+        }
         // row normaliser from the segment partials: lane g holds segment g (S <= 8), fixed reduction order
         float lse;
         {
-            const float mg = lane < S ? part.m[r * S + lane] : neg_inf();
             const float M = warp_max(mg);
-            const float term = mg != neg_inf() ? part.s[r * S + lane] * expf(mg - M) : 0.f;
-            const float sum = warp_sum(term);
+            const float sum = warp_sum(mg != neg_inf() ? sg * expf(mg - M) : 0.f);
             lse = M == neg_inf() ? neg_inf() : M + logf(sum);
         }
         if (lane == 0) row_lse[r] = lse;
-        if (lse_in) lse = lse_in[r];
+        if (lse_in) lse = lse_given;
         if (lane == 0) s_lse[h] = lse;
         const float parent = s_parent[h];
         const bool eos_ok = s_eos_ok[h] != 0;
 
         // the row's K1 largest raw logits, merged over segments, as keys in `merged`
-        if (S == 1) {
-            for (int e = lane; e < K1; e += 32) {
-                const int ix = part.top_idx[(int64_t)r * K1 + e];
-                merged[e] = ix >= 0 ? row_key(part.top_val[(int64_t)r * K1 + e], ix) : 0ull;
-            }
-        } else {
-            const int n = S * K1;
+        if (S > 1) {
+            const int n = n_ent;
             for (int e = lane; e < K1; e += 32) merged[e] = 0ull;
-            for (int e = lane; e < n; e += 32) {
-                const int ix = part.top_idx[(int64_t)r * n + e];
-                stage[e] = ix >= 0 ? row_key(part.top_val[(int64_t)r * n + e], ix) : 0ull;
-            }
             __syncwarp();
             // every segment's list is in descending key order (empty entries, key 0, last): the place of an
             // entry in the merged order is its place in its own list plus, for every other list, the number of
@@ -335,7 +307,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         //      raise its met count by one.  They all land in the same bank, so of one row at most k can ever be
         //      kept: with more, only the row's k best go on (the rest could not be selected; the bank still
         //      counts at least k candidates, which is all the allocation needs to know).
-        for (int h = warp - 1; h < k; h += kCandWarps - 1) {
+        for (int h = warp - 1; h < k; h += n_warps - 1) {
             if (s_kind[h] != 1) continue;
             const uint64_t m = s_mask[h]; const int a = s_active[h];
             const float lse = s_lse[h], parent = s_parent[h];
@@ -348,8 +320,9 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
                     if (a >= 0) ok = j == a + 1;
                     else {
                         ok = ((sc.first_mask >> j) & 1ull) && !((m >> j) & 1ull);
-                        uint64_t earlier = ok ? sc.first_mask & ~m & ((1ull << j) - 1ull) : 0ull;   // same token earlier?
-                        while (earlier) { const int e = __ffsll((long long)earlier) - 1; ok = ok && sc.ctok[e] != sc.ctok[j]; earlier &= earlier - 1; }
+                        // the same token may open an earlier word/phrase that is still unmet: then that one is listed
+                        for (int e = ok ? sc.prev_same[j] : 255; e != 255; e = sc.prev_same[e])
+                            if (!((m >> e) & 1ull)) { ok = false; break; }
                     }
                 }
                 float x = neg_inf();
@@ -392,15 +365,54 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     // ---- sources 1 and 3 with their updated constraint marks; cells that advance a hypothesis through
     //      its constraints are left to source 2, which lists every such cell (no duplicates arise) ----------
     const int ns1 = s_ns1;
-    for (int t = tid; t < 2 * k; t += kCandThreads) {
+    // constraints[h].add(w) (Section 3.1, last paragraph) for these at most 2k cells: continue the begun phrase
+    // if w is its next token; otherwise reset that phrase's marks and let w open the first wholly unmet
+    // word/phrase it matches.  The scan over the constraint positions is spread over the CTA.
+    // Step 1: continue the begun phrase, or unwind it; note the marks that remain.
+    __shared__ uint64_t a_mask[2 * kMaxK];     // marks after a possible unwind (before w opens anything)
+    __shared__ int a_w[2 * kMaxK];             // the token, -1: no cell / nothing to look for
+    __shared__ int a_pos[2 * kMaxK];           // lowest position w can open (64: none)
+    for (int t = tid; t < 2 * k; t += n_threads) {
+        int h, i; bool have = true;
+        if (t < k) { have = t < ns1; h = have ? s1_h[t] : 0; i = have ? s1_i[t] : 0; }
+        else { h = t - k; i = 0; have = rt_n[h] != 0 && rt_ptr[h] == 0; }      // else: best cell already in source 1
+        a_pos[t] = 64; a_w[t] = -1;
+        if (have && s_kind[h] == 1) {
+            const int w = rt_w[h * k + i];
+            uint64_t m = s_mask[h]; const int a = s_active[h];
+            if (a >= 0 && w != sc.ctok[a + 1]) {                                 // the begun phrase is broken: unwind
+                const int p0 = sc.pstart[a];
+                m &= ~(((2ull << a) - 1ull) & ~((1ull << p0) - 1ull));
+            }
+            a_mask[t] = m;
+            if (!(a >= 0 && w == sc.ctok[a + 1])) a_w[t] = w;                    // otherwise it simply continues
+        }
+    }
+    __syncthreads();
+    // Step 2: the first wholly unmet word/phrase that w opens, if any.
+    for (int q = tid; q < 2 * k * kMaxC; q += n_threads) {
+        const int t = q >> 6, j = q & 63;
+        const int w = a_w[t];
+        if (w >= 0 && j < C && sc.ctok[j] == w && ((sc.first_mask & ~a_mask[t]) >> j) & 1ull) atomicMin(&a_pos[t], j);
+    }
+    __syncthreads();
+    // Step 3: finish the update; cells that raise the met count belong to source 2 and are skipped here.
+    for (int t = tid; t < 2 * k; t += n_threads) {
         int h, i;
         if (t < k) { if (t >= ns1) continue; h = s1_h[t]; i = s1_i[t]; }
-        else { h = t - k; i = 0; if (rt_n[h] == 0 || rt_ptr[h] > 0) continue; }   // best cell already in source 1
+        else { h = t - k; i = 0; if (rt_n[h] == 0 || rt_ptr[h] > 0) continue; }
         const int w = rt_w[h * k + i];
         uint64_t m = s_mask[h]; int a = s_active[h];
         if (s_kind[h] == 1) {
             const int before = __popcll(m);
-            cons_add(sc, m, a, w);
+            if (a >= 0 && w == sc.ctok[a + 1]) {
+                const int nn = a + 1;
+                m |= 1ull << nn; a = ((sc.last_mask >> nn) & 1ull) ? -1 : nn;
+            } else {
+                m = a_mask[t]; a = -1;
+                const int j = a_pos[t];
+                if (j < 64) { m |= 1ull << j; a = ((sc.last_mask >> j) & 1ull) ? -1 : j; }
+            }
             if (__popcll(m) == before + 1) continue;
         }
         const int slot = atomicAdd(&s_ncand, 1);
@@ -416,7 +428,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     // ---- group by bank, order inside each bank (Section 3.1): order (bank asc, score desc, flat asc) ---------
     int n_sort = 32;
     while (n_sort < n) n_sort <<= 1;
-    for (int i = tid; i < n_sort; i += kCandThreads) {
+    for (int i = tid; i < n_sort; i += n_threads) {
         SortEnt e;
         if (i < n) {
             e.hi = ((uint64_t)__popcll(c_mask[i]) << 32) | (uint32_t)(0xffffffffu - ord32(c_score[i]));
@@ -425,11 +437,12 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         ent[i] = e;
     }
     __syncthreads();
-    if (n <= kCandThreads) {
+    if (n <= 160) {
         // short list: every thread counts how many entries precede its own (keys are distinct) and writes it there
         if (tid < n) {
             const SortEnt me = ent[tid];
             int rank = 0;
+#pragma unroll 4
             for (int j = 0; j < n; ++j) {
                 const SortEnt o = ent[j];
                 rank += o.hi < me.hi || (o.hi == me.hi && o.lo < me.lo);
@@ -437,10 +450,37 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
             Cand c; c.score = c_score[tid]; c.flat = c_flat[tid]; c.mask = c_mask[tid]; c.active = c_active[tid]; c.pad_ = 0;
             cand_out[(int64_t)b * d.max_cand + rank] = c;
         }
+    } else if (n_sort <= n_threads) {
+        // medium list: bitonic network with one entry per thread; partners less than a warp apart are reached by
+        // shuffles, the others through shared memory
+        SortEnt me = ent[tid < n_sort ? tid : 0];
+        for (int size = 2; size <= n_sort; size <<= 1) {
+            for (int str = size >> 1; str > 0; str >>= 1) {
+                SortEnt o;
+                if (str >= 32) {
+                    __syncthreads();
+                    if (tid < n_sort) ent[tid] = me;
+                    __syncthreads();
+                    o = ent[(tid ^ str) < n_sort ? (tid ^ str) : 0];
+                } else if (tid < n_sort) {                      // (whole warps: n_sort is a multiple of 32)
+                    o.hi = __shfl_xor_sync(kFullMask, me.hi, str);
+                    o.lo = __shfl_xor_sync(kFullMask, me.lo, str);
+                    o.id = __shfl_xor_sync(kFullMask, me.id, str);
+                } else o = me;
+                const bool mine_first = me.hi < o.hi || (me.hi == o.hi && me.lo < o.lo);
+                const bool want_first = ((tid & str) == 0) == ((tid & size) == 0);     // keep the smaller of the pair?
+                if (mine_first != want_first) me = o;
+            }
+        }
+        if (tid < n) {
+            const int id = me.id;
+            Cand c; c.score = c_score[id]; c.flat = c_flat[id]; c.mask = c_mask[id]; c.active = c_active[id]; c.pad_ = 0;
+            cand_out[(int64_t)b * d.max_cand + tid] = c;
+        }
     } else {
         for (int size = 2; size <= n_sort; size <<= 1) {
             for (int str = size >> 1; str > 0; str >>= 1) {
-                for (int t = tid; t < n_sort / 2; t += kCandThreads) {
+                for (int t = tid; t < n_sort / 2; t += n_threads) {
                     const int pos = 2 * t - (t & (str - 1));
                     SortEnt a = ent[pos], c = ent[pos + str];
                     const bool gt = a.hi > c.hi || (a.hi == c.hi && a.lo > c.lo);
@@ -450,7 +490,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
                 __syncthreads();
             }
         }
-        for (int i = tid; i < n; i += kCandThreads) {
+        for (int i = tid; i < n; i += n_threads) {
             const int id = ent[i].id;
             Cand c; c.score = c_score[id]; c.flat = c_flat[id]; c.mask = c_mask[id]; c.active = c_active[id]; c.pad_ = 0;
             cand_out[(int64_t)b * d.max_cand + i] = c;
@@ -462,20 +502,39 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
 
 }  // namespace
 
-size_t candidates_smem_bytes(const Dims& d) { return (size_t)make_layout(d.k, d.K1, d.S, d.max_cand).total; }
+// Threads per CTA: 1024 when every sentence gets an SM of its own (then only the latency of one CTA counts),
+// 512 otherwise (two CTAs fit an SM's registers); fewer if the per-warp scratch would not fit shared memory.
+static size_t g_smem_limit = 48 * 1024;     // raised by configure_candidates
+static int g_sm_count = 1;
+static int pick_threads(const Dims& d, size_t smem_limit) {
+    for (int t = d.B <= g_sm_count ? kCandMaxThreads : kCandMaxThreads / 2; t > 256; t >>= 1)
+        if ((size_t)make_layout(d.k, d.K1, d.S, d.max_cand, t / 32).total <= smem_limit) return t;
+    return 256;
+}
+
+size_t candidates_smem_bytes(const Dims& d) { return (size_t)make_layout(d.k, d.K1, d.S, d.max_cand, 256 / 32).total; }
 
 cudaError_t configure_candidates(const Dims& d) {
+    int dev = 0, lim = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&lim, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return e;
+    g_smem_limit = (size_t)lim;
+    e = cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const int t = pick_threads(d, g_smem_limit);
     return cudaFuncSetAttribute(candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)candidates_smem_bytes(d));
+                                make_layout(d.k, d.K1, d.S, d.max_cand, t / 32).total);
 }
 
 cudaError_t launch_candidates(const void* logits, int64_t stride, const Dims& d, const SentCons* cons,
                               const Beam& cur, const ScanOut& part, const float* lse_in, float* row_lse,
                               Cand* cand, int32_t* ncand, int32_t* bank_count, uint32_t* status,
                               int32_t* open_count, cudaStream_t st, int* launches) {
-    const size_t smem = candidates_smem_bytes(d);
-    candidates_kernel<<<d.B, kCandThreads, smem, st>>>(logits, stride, d, cons, cur, part, lse_in, row_lse, cand,
-                                                      ncand, bank_count, status, open_count);
+    const int threads = pick_threads(d, g_smem_limit);
+    const size_t smem = (size_t)make_layout(d.k, d.K1, d.S, d.max_cand, threads / 32).total;
+    candidates_kernel<<<d.B, threads, smem, st>>>(logits, stride, d, cons, cur, part, lse_in, row_lse, cand,
+                                                  ncand, bank_count, status, open_count);
     ++*launches;
     return cudaGetLastError();
 }

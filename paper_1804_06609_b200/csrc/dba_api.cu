@@ -98,6 +98,12 @@ dba_status check_config(const dba_config* c, Shape* shape, std::vector<SentCons>
                 if (i == tb - 1) sc.last_mask |= 1ull << j;
             }
         }
+        for (int q = 0; q < j; ++q) {
+            sc.prev_same[q] = 255;
+            if (!((sc.first_mask >> q) & 1ull)) continue;
+            for (int e = q - 1; e >= 0; --e)
+                if (((sc.first_mask >> e) & 1ull) && sc.ctok[e] == sc.ctok[q]) { sc.prev_same[q] = (uint8_t)e; break; }
+        }
         sc.C = j;
         sc.n_phrases = pb - pa;
         if (shape && sc.n_phrases > shape->max_phrases) shape->max_phrases = sc.n_phrases;

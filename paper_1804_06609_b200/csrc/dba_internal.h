@@ -25,6 +25,7 @@ struct SentCons {
     uint64_t last_mask;    // bit j: position j closes its word/phrase
     int32_t ctok[kMaxC];
     uint8_t pstart[kMaxC]; // first position of the phrase position j belongs to
+    uint8_t prev_same[kMaxC]; // nearest earlier phrase-opening position with the same token (255: none)
 };
 
 // One beam (all sentences): arrays of R = B*k entries.

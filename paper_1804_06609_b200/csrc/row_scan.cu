@@ -124,7 +124,7 @@ void plan_segments(Dims& d, int sm_count) {
     int chunks = 8;
     auto segs = [&](int c) { return (d.V + c * chunk_elems - 1) / (c * chunk_elems); };
     while (segs(chunks) > kMaxSeg) chunks *= 2;                       // very long rows: longer segments
-    while (chunks > 1 && (int64_t)d.R * segs(chunks) < 6LL * sm_count && segs(chunks / 2) <= kMaxSeg) chunks /= 2;
+    while (chunks > 1 && (int64_t)d.R * segs(chunks) < 4LL * sm_count && segs(chunks / 2) <= kMaxSeg) chunks /= 2;
     d.seg_len = chunks * chunk_elems;
     d.S = segs(chunks);
     d.K1 = d.k + 2;
