@@ -7,7 +7,7 @@ namespace dba {
 
 namespace {
 
-constexpr int kAllocWarps = 4;       // sentences per CTA
+constexpr int kAllocWarps = 1;       // sentences per CTA
 constexpr int kBanks = kMaxC + 1;
 
 // Nearest bank above / below b whose bit is set in the 65-bit set (lo: banks 0..63, hi: bank 64); -1 if none.
@@ -41,31 +41,52 @@ allocate_kernel(Dims d, const SentCons* __restrict__ cons, Beam cur, Beam nxt, c
     const int C = cons[b].C;
     int* n = s_n[warp]; int* alloc = s_alloc[warp]; int* off = s_off[warp]; int* sel = s_sel[warp];
 
-    // bank sizes; equal base share, remainder to the top bank C (Section 3.2)
+    // Lane l looks after banks l, l + 32 and l + 64 (there are at most 65).
+    // bank sizes; equal base share, remainder to the top bank C (Section 3.2); offsets of the banks inside the
+    // bank-ordered candidate list
     const int share = k / (C + 1);
-    for (int q = lane; q <= C; q += 32) {
-        n[q] = bank_count[b * kBanks + q];
-        alloc[q] = share + (q == C ? k - share * (C + 1) : 0);
+    int nq[3], aq[3];
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+        const int q = lane + 32 * j;
+        nq[j] = q <= C ? bank_count[b * kBanks + q] : 0;
+        aq[j] = q <= C ? share + (q == C ? k - share * (C + 1) : 0) : 0;
     }
-    __syncwarp();
-    if (lane == 0) {
-        // exclusive offsets of the banks inside the bank-ordered candidate list
-        int acc = 0;
-        for (int q = 0; q <= C; ++q) { off[q] = acc; acc += n[q]; }
-        if (d.flags & DBA_FLAG_ADJUST_OFF) {
-            for (int q = 0; q <= C; ++q) alloc[q] = min(alloc[q], n[q]);
-        } else {
-            // Adjustment: every bank with more slots than candidates passes the surplus to the nearest
-            // banks that have more candidates than slots, the higher one first at equal distance.
-            uint64_t over_lo = 0, need_lo = 0; bool over_hi = false, need_hi = false;
-            for (int q = 0; q <= C; ++q) {
-                const bool ov = alloc[q] > n[q], nd = n[q] > alloc[q];
-                if (q < 64) { over_lo |= (uint64_t)ov << q; need_lo |= (uint64_t)nd << q; }
-                else { over_hi = ov; need_hi = nd; }
-            }
-            for (int q = 0; q <= C; ++q) {
-                const bool ov = q < 64 ? ((over_lo >> q) & 1ull) : over_hi;
-                if (!ov) continue;
+    {
+        int run = 0;                                  // exclusive prefix of n over banks, 32 at a time
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+            int incl = nq[j];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(kFullMask, incl, o); if (lane >= o) incl += t; }
+            const int q = lane + 32 * j;
+            if (q <= C) { off[q] = run + incl - nq[j]; n[q] = nq[j]; }
+            run += __shfl_sync(kFullMask, incl, 31);
+        }
+    }
+    if (d.flags & DBA_FLAG_ADJUST_OFF) {
+#pragma unroll
+        for (int j = 0; j < 3; ++j) { const int q = lane + 32 * j; if (q <= C) alloc[q] = min(aq[j], nq[j]); }
+        __syncwarp();
+    } else {
+        // Adjustment: every bank with more slots than candidates passes the surplus to the nearest banks that
+        // have more candidates than slots, the higher one first at equal distance.  The sets of such banks are
+        // bit masks (banks 0..63 in a 64-bit word, bank 64 apart); the walk itself is short and serial.
+        const unsigned o0 = __ballot_sync(kFullMask, aq[0] > nq[0]), o1 = __ballot_sync(kFullMask, aq[1] > nq[1]);
+        const unsigned d0 = __ballot_sync(kFullMask, nq[0] > aq[0]), d1 = __ballot_sync(kFullMask, nq[1] > aq[1]);
+        const bool over_hi = __any_sync(kFullMask, lane == 0 && aq[2] > nq[2]);
+        bool need_hi = __any_sync(kFullMask, lane == 0 && nq[2] > aq[2]);
+        const uint64_t over_lo = (uint64_t)o0 | ((uint64_t)o1 << 32);
+        uint64_t need_lo = (uint64_t)d0 | ((uint64_t)d1 << 32);
+#pragma unroll
+        for (int j = 0; j < 3; ++j) { const int q = lane + 32 * j; if (q <= C) alloc[q] = aq[j]; }
+        __syncwarp();
+        if (lane == 0) {
+            uint64_t todo = over_lo;
+            bool todo_hi = over_hi;
+            while (todo || todo_hi) {
+                int q;
+                if (todo) { q = __ffsll((long long)todo) - 1; todo &= todo - 1; } else { q = 64; todo_hi = false; }
                 int surplus = alloc[q] - n[q];
                 alloc[q] = n[q];
                 while (surplus > 0) {
@@ -80,12 +101,27 @@ allocate_kernel(Dims d, const SentCons* __restrict__ cons, Beam cur, Beam nxt, c
                 }
             }
         }
-        // the best alloc[q] candidates of every bank (they are ordered inside the bank already)
-        int ns = 0;
-        for (int q = 0; q <= C; ++q)
-            for (int i = 0; i < alloc[q]; ++i) sel[ns++] = off[q] + i;
-        off[0] = ns;   // reuse as the selected count
+        __syncwarp();
     }
+    // the best alloc[q] candidates of every bank (they are ordered inside the bank already)
+    int ns_total;
+    {
+        int run = 0;
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+            const int q = lane + 32 * j;
+            const int a = q <= C ? alloc[q] : 0;
+            int incl = a;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(kFullMask, incl, o); if (lane >= o) incl += t; }
+            const int first = run + incl - a;
+            for (int i = 0; i < a; ++i) sel[first + i] = off[q] + i;
+            run += __shfl_sync(kFullMask, incl, 31);
+        }
+        ns_total = run;
+    }
+    __syncwarp();
+    if (lane == 0) off[0] = ns_total;   // (kept where the code below reads it)
     __syncwarp();
     const int ns = off[0];
     const Cand* cb = cand + (int64_t)b * d.max_cand;
