@@ -15,6 +15,8 @@ constexpr int kMaxSeg = 8;         // row segments scanned by different CTAs
 // device status word bits (sticky; read by dba_finalize)
 constexpr uint32_t kStatusTimeout = 1u;    // a bounded wait on an mbarrier gave up
 constexpr uint32_t kStatusOverflow = 2u;   // an internal list ran out of room (results of that step invalid)
+// further words of the status block: counters (diagnostics, never an error)
+constexpr int kStatusWordRescans = 1;      // row segments the scan kernel had to rank from global memory again
 
 // Per-sentence constraint table, phrases flattened to token positions 0..C-1 (Section 3 of the paper:
 // the constraint count is the total number of tokens over all words and phrases).

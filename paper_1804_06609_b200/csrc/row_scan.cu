@@ -117,14 +117,20 @@ __global__ void row_merge_kernel(int R, int S, int K1, int n_top, const float* _
 }  // namespace
 
 void plan_segments(Dims& d, int sm_count) {
-    // Segments are 1, 2, 4 or 8 chunks of 8 KB; shorter segments when there are few rows, so that every SM
-    // has several (row, segment) items to work on, but never more than kMaxSeg segments per row.
+    // Segments are whole 4 KB chunks, at most twelve of them (what one team of the streaming kernel holds);
+    // shorter segments when there are few rows, so that every SM has several (row, segment) items to work on,
+    // but never more than kMaxSeg segments per row.
     const int es = d.dtype == DBA_F32 ? 4 : 2;
-    const int chunk_elems = 8192 / es;
-    int chunks = 8;
-    auto segs = [&](int c) { return (d.V + c * chunk_elems - 1) / (c * chunk_elems); };
+    const int chunk_elems = 4096 / es;
+    const int row_chunks = (d.V + chunk_elems - 1) / chunk_elems;
+    auto segs = [&](int c) { return (row_chunks + c - 1) / c; };
+    int chunks = 12;
     while (segs(chunks) > kMaxSeg) chunks *= 2;                       // very long rows: longer segments
-    while (chunks > 1 && (int64_t)d.R * segs(chunks) < 4LL * sm_count && segs(chunks / 2) <= kMaxSeg) chunks /= 2;
+    if (chunks == 12) {
+        chunks = (row_chunks + segs(12) - 1) / segs(12);             // same number of segments, evened out
+        while (chunks > 1 && (int64_t)d.R * segs(chunks) < 4LL * sm_count && segs((chunks + 1) / 2) <= kMaxSeg)
+            chunks = (chunks + 1) / 2;
+    }
     d.seg_len = chunks * chunk_elems;
     d.S = segs(chunks);
     d.K1 = d.k + 2;
