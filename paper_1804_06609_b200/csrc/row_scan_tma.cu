@@ -40,12 +40,11 @@ constexpr int kTeamWarps = 11;                 // consumer warps per team = most
 constexpr int kTeams = 2;                      // teams take alternate items
 constexpr int kNC = kTeams * kTeamWarps;       // consumer warps
 constexpr int kSlots = 4;                      // items in flight: buffers (176 KB in all) and selection state
-constexpr int kNR = kSlots;                    // selector warps, one per slot
-// The selectors come first: their work is a chain of dependent steps on the critical path of an item, and
-// the warp scheduler favours the warps that come first when several are ready.
-constexpr int kWarpRank = 0;                   // first selector warp
-constexpr int kWarpProd = kNR;                 // the producer's warp
-constexpr int kWarpCons = kNR + 1;             // first consumer warp
+constexpr int kNR = kSlots;                    // selector warps (and ranking warps), one per slot
+constexpr int kWarpSel = 0;                    // first selector warp
+constexpr int kWarpRank = kNR;                 // first ranking warp
+constexpr int kWarpProd = 2 * kNR;             // the producer's warp
+constexpr int kWarpCons = 2 * kNR + 1;         // first consumer warp
 constexpr int kThreads = 32 * (kWarpCons + kNC);
 constexpr int kHitCap = 96;                    // cells reaching the bound that one item may have
 constexpr int kKeyCap = 128;                   // entries at or above the bound that one item may hold
@@ -66,8 +65,12 @@ struct Smem {
     uint32_t lane_key[kSlots][kTeamWarps][32];              // lane maxima as ordered integers
     float warp_sum[kSlots][2][kTeamWarps];  // alternate uses of a slot take alternate halves
     float warp_ref[kSlots][2][kTeamWarps];  // the whole number c of exp2(x*log2e - c) each warp used (-inf: no data)
+    uint64_t hits_ready[kSlots];            // the selector has left the item's cell list
+    uint64_t ranked[kSlots];                // the ranking warp is done with the item
     int hit_lane[kNR][kHitCap];             // lanes that reach the bound: chunk * 32 + lane
-    int hit[kNR][kHitCap];                  // cells that reach the bound: (first vector of the pair) * 2 + parity
+    int hit[kSlots][2][kHitCap];            // cells that reach the bound: (first vector of the pair) * 2 + parity
+    int hit_n[kSlots][2];                   // how many (above kHitCap: the list overflowed)
+    float hit_bound[kSlots][2];
     int abort_flag;
 };
 
@@ -246,7 +249,6 @@ struct ItemIter {
     __device__ int seg() const { return seg_; }
     __device__ int bytes() const { return bytes_; }
     __device__ int n_chunks() const { return n_chunks_; }
-    __device__ uint32_t team() const { return n_item % kTeams; }
     __device__ uint32_t slot() const { return n_item % kSlots; }
     __device__ uint32_t use() const { return n_item / kSlots; }            // how often the slot was used before
     __device__ uint32_t slot_phase() const { return use() & 1u; }
@@ -300,6 +302,7 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
             mbar_init(smem_u32(&sm.full[s]), 1); mbar_init(smem_u32(&sm.loaded[s]), kTeamWarps);
             mbar_init(smem_u32(&sm.reports_in[s]), kTeamWarps); mbar_init(smem_u32(&sm.slot_free[s]), 1);
             mbar_init(smem_u32(&sm.sums_in[s][0]), kTeamWarps); mbar_init(smem_u32(&sm.sums_in[s][1]), kTeamWarps);
+            mbar_init(smem_u32(&sm.hits_ready[s]), 1); mbar_init(smem_u32(&sm.ranked[s]), 1);
         }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -332,8 +335,8 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
     } else if (warp >= kWarpCons) {
         // ------------------------------------------------------------------ consumers
         const int team = (warp - kWarpCons) / kTeamWarps, chunk = (warp - kWarpCons) - team * kTeamWarps;
-#pragma unroll 1
         ItemIter it(p, (int)sizeof(T));
+#pragma unroll 1
         for (it.skip(team); it.valid(); it.skip(kTeams)) {
             const uint32_t slot = it.slot(), half = it.use() & 1u;
             const int nvec = chunk < it.n_chunks() ? it.chunk_vecs(chunk) : 0;
@@ -395,20 +398,18 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
                 mbar_arrive(smem_u32(&sm.sums_in[slot][half]));
             }
         }
-    } else {
+    } else if (warp < kWarpRank) {
         // ------------------------------------------------------------------ selector of slot rk
-        const int rk = warp - kWarpRank;
+        const int rk = warp - kWarpSel;
         const uint32_t slot = (uint32_t)rk;
-        uint64_t* keys = sm.key[rk];
-        int* hits = sm.hit[rk];
         ItemIter it(p, (int)sizeof(T));
         it.skip(rk);                                      // this selector's first item
 #pragma unroll 1
         while (it.valid()) {
-            const int row = it.row(p.open_list);          // needed late, asked for early
             if (!mbar_wait_warp(smem_u32(&sm.reports_in[slot]), it.slot_phase(), abort_flag)) break;
             // The bound: the K1-th largest report, i.e. the largest report that at least K1 reports reach.
-            const uint32_t half = it.use() & 1u, use_phase = (it.use() >> 1) & 1u;
+            const uint32_t half = it.use() & 1u;
+            int* hits = sm.hit[slot][half];
             const int tap = it.report_tap(p.K1);
             const int n_rep = tap < 0 ? 0 : it.report_warps() << (5 - tap);     // a multiple of four
             uint32_t best = 0;
@@ -504,10 +505,35 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
                 }
                 listed = nh <= kHitCap;
             }
+            if (lane == 0) { sm.hit_n[slot][half] = listed ? nh : kHitCap + 1; sm.hit_bound[slot][half] = tau; }
+            // The ranking warp must be done with the slot's previous item: then it has seen the previous list
+            // being announced, and has read the sums that the team's next item will overwrite.
+            if (!mbar_wait_warp(smem_u32(&sm.ranked[slot]), it.slot_phase() ^ 1u, abort_flag)) break;
             // nothing of the slot's shared maxima and reports is needed any more: let the team's next item in
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sm.slot_free[slot]));
-
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&sm.slot_free[slot]));
+                mbar_arrive(smem_u32(&sm.hits_ready[slot]));
+            }
+            it.skip(kSlots);
+        }
+    } else {
+        // ------------------------------------------------------------------ ranking warp of slot rk
+        const int rk = warp - kWarpRank;
+        const uint32_t slot = (uint32_t)rk;
+        uint64_t* keys = sm.key[rk];
+        ItemIter it(p, (int)sizeof(T));
+        it.skip(rk);
+#pragma unroll 1
+        while (it.valid()) {
+            const int row = it.row(p.open_list);
+            const uint32_t half = it.use() & 1u, use_phase = (it.use() >> 1) & 1u;
+            const int nc = it.n_chunks();
+            if (!mbar_wait_warp(smem_u32(&sm.hits_ready[slot]), it.slot_phase(), abort_flag)) break;
+            const int* hits = sm.hit[slot][half];
+            const int nh = sm.hit_n[slot][half];
+            const float tau = sm.hit_bound[slot][half];
+            bool listed = nh <= kHitCap;
             const int elem0 = it.seg() * p.seg_len, n_elem = it.bytes() / (int)sizeof(T);
             const T* src = (const T*)p.logits + (int64_t)row * p.stride + elem0;
             int n = 0;
@@ -593,6 +619,7 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
                 rank_from_global<T>((const T*)p.logits + (int64_t)row * p.stride, elem0, elem0 + n_elem, p.K1, tv, ti);
             }
             __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm.ranked[slot]));
             it.skip(kSlots);
         }
     }
