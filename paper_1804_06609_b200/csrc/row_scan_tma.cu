@@ -4,11 +4,11 @@
 // items are in flight, each with a shared-memory buffer and a selector warp of its own.  Warps have fixed
 // roles and talk through mbarriers only (no CTA-wide barrier inside the loop); a consumer never waits for
 // another consumer:
-//   producer    one thread refills a buffer as soon as the item in it has been copied to registers: one bulk
+//   producer    one thread refills a buffer as soon as the item's consumers are done with it: one bulk
 //               asynchronous copy (TMA, cp.async.bulk) per item;
 //   consumers   two teams of eleven warps, the teams taking alternate items.  A warp owns one chunk of its
-//               item: it copies the chunk into registers (eight 16-byte vectors per lane), takes maxima, and
-//               sums exp2(x*log2e - c) (Section 2's normaliser) with c a whole number at or above the warp's
+//               item: it reads the chunk (eight 16-byte vectors per lane) once for the maxima and once more for
+//               the sum of exp2(x*log2e - c) (Section 2's normaliser), c a whole number at or above the warp's
 //               maximum.  The selection piggybacks on the maxima: the maxima of every pair of vectors (cells
 //               of eight entries) and of every lane go to shared memory as they are, and the butterfly that
 //               gives the warp's maximum is tapped midway, which yields the maxima of G groups of lanes
@@ -356,9 +356,7 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
                         v[i] = i * 32 + lane < nvec ? vec[i * 32] : make_uint4(w, w, w, w);   // beyond the row: -inf
                     }
                 }
-                __syncwarp();
             }
-            if (lane == 0) mbar_arrive(smem_u32(&sm.loaded[slot]));         // this warp's chunk lives in registers now
             if (nvec > 0) {
 #pragma unroll
                 for (int q = 0; q < kPairs; ++q) pmax[q] = Vec<T>::max2(Vec<T>::vec_max(v[2 * q]), Vec<T>::vec_max(v[2 * q + 1]));
@@ -386,12 +384,21 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
                 cref = ceilf(wm * kLog2e);            // a whole number: rescaling by powers of two is exact
                 const uint64_t L2 = pack2(kLog2e, kLog2e), C2 = pack2(-cref, -cref);
                 uint64_t a0 = 0, a1 = 0;
+                // the chunk is read from the buffer a second time: held in registers since the maxima, it would
+                // leave the exponentials too few registers to overlap one another
+                const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[slot]) + chunk * kChunkVecs + lane;
 #pragma unroll
-                for (int i = 0; i < kVecsPerLane; ++i) Vec<T>::exp_sum(v[i], L2, C2, a0, a1);
+                for (int i = 0; i < kVecsPerLane; ++i) {
+                    const uint32_t w = Vec<T>::kNegInfWord;
+                    const uint4 vv = i * 32 + lane < nvec ? vec[i * 32] : make_uint4(w, w, w, w);
+                    Vec<T>::exp_sum(vv, L2, C2, a0, a1);
+                }
                 float s0, s1, s2, s3;
                 unpack2(a0, s0, s1); unpack2(a1, s2, s3);
                 ssum = (s0 + s1) + (s2 + s3);
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm.loaded[slot]));         // this warp is done with the buffer
             const float wsum = warp_sum(ssum);
             if (lane == 0) {
                 sm.warp_sum[slot][half][chunk] = wsum; sm.warp_ref[slot][half][chunk] = cref;
