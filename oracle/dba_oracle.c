@@ -24,6 +24,10 @@
  *                               paper only outlines the procedure and the figure that shows one is lost)
  *   finishing          pinned   every completed output holds all constraints; exhaustive regime
  *                               equals brute force over all sequences
+ *   pruning, stopping  pinned   closed form on a two-word vocabulary (two scores exactly theta' apart: kept iff
+ *                               theta' <= threshold), the best completed hypothesis is never removed, an
+ *                               infinite threshold changes nothing, stop bits on hand-built beams;
+ *                               parity unpinned: which score is compared (READING below)
  *   conventions        parity unpinned: finished hypotheses staying on the beam with a frozen
  *                               score, empty slots, global order of the new beam, length counted
  *                               with the end token (READINGS below)
@@ -50,6 +54,7 @@ typedef struct {
 typedef struct orc_sentence {
     int k, V, max_steps, pad, bos, eos;
     unsigned flags;
+    float prune;       /* Section 4's pruning threshold; <= 0: no pruning */
     /* constraints flattened to positions 0..C-1 (Section 3: C = total tokens over all words and phrases) */
     int C;
     int ctok[ORC_MAX_C];
@@ -427,6 +432,23 @@ int orc_step(orc_sentence *s, const void *logits, int dtype, long row_stride, fl
        (READING: one global order, not bank by bank). */
     sort_cands(kept, nkept, V);
 
+    /* Section 4 (and Section 6.3): threshold pruning of the beam.  A hypothesis whose log-probability is not
+       within the threshold of the best completed hypothesis is removed, whether it is itself complete or not.
+       READING: both sides of the comparison are cumulative log-probabilities (the scores the beam is ordered
+       by); a removed hypothesis leaves an empty slot; the beam is in decreasing order, so they are its tail. */
+    if (s->prune > 0) {
+        float best = -INFINITY;
+        for (int i = 0; i < nkept; ++i)
+            if (kept[i].w == s->eos && kept[i].score > best) best = kept[i].score;
+        if (best != -INFINITY) {
+            volatile float cut = best - s->prune;
+            int n = 0;
+            for (int i = 0; i < nkept; ++i)
+                if (!(kept[i].score < cut)) kept[n++] = kept[i];
+            nkept = n;
+        }
+    }
+
     int *hb = s->hist_bp + (size_t)s->t * k, *ht = s->hist_tok + (size_t)s->t * k;
     for (int i = 0; i < k; ++i) {
         if (i < nkept) {
@@ -442,6 +464,26 @@ int orc_step(orc_sentence *s, const void *logits, int dtype, long row_stride, fl
     s->t++;
     free(kept); free(tmp); free(S); free(lse);
     return 0;
+}
+
+/* Section 4's pruning threshold ("within 20" in the paper's experiments); <= 0 switches pruning off. */
+void orc_set_prune(orc_sentence *s, float threshold) { s->prune = threshold; }
+
+/* ------------------------------------------------------------------------------------------
+ * Section 4: "Decoding stops when either all hypotheses still on the beam are completed or the maximum
+ * length is reached"; Section 6.4's alternative, early stopping, stops at the first completed hypothesis.
+ * Bit 0: the beam is not empty and every hypothesis on it is completed.  Bit 1: some hypothesis on the
+ * beam is completed.  The caller owns the loop and decides which to act on.
+ * ------------------------------------------------------------------------------------------ */
+int orc_stop_flags(const orc_sentence *s)
+{
+    int live = 0, done = 0;
+    for (int h = 0; h < s->k; ++h) {
+        if (isinf(s->score[h])) continue;
+        ++live;
+        if (s->tok[h] == s->eos) ++done;
+    }
+    return (live > 0 && done == live ? 1 : 0) | (done > 0 ? 2 : 0);
 }
 
 /* ------------------------------------------------------------------------------------------

@@ -53,6 +53,9 @@ def lib():
         L.orc_last_allocation.argtypes = [C.c_void_p, i32p, i32p]
         L.orc_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_long, f32p]
         L.orc_finalize.argtypes = [C.c_void_p, i32p, i32p, f32p, i32p]
+        L.orc_set_prune.argtypes = [C.c_void_p, C.c_float]
+        L.orc_set_prune.restype = None
+        L.orc_stop_flags.argtypes = [C.c_void_p]
         _lib = L
     return _lib
 
@@ -89,7 +92,7 @@ def allocate(k: int, n, flags: int = 0) -> np.ndarray:
 class Sentence:
     """One sentence's constrained beam: constraints are a list of phrases (lists of token ids)."""
 
-    def __init__(self, k, V, max_steps, phrases, pad=0, bos=1, eos=2, flags=0):
+    def __init__(self, k, V, max_steps, phrases, pad=0, bos=1, eos=2, flags=0, prune=0.0):
         self.k, self.V, self.max_steps = k, V, max_steps
         self.pad, self.bos, self.eos, self.flags = pad, bos, eos, flags
         off = np.zeros(len(phrases) + 1, dtype=np.int32)
@@ -101,6 +104,8 @@ class Sentence:
         if not self._h:
             raise ValueError("oracle rejected the constraint set")
         self.C = lib().orc_num_constraints(self._h)
+        if prune > 0:
+            lib().orc_set_prune(self._h, prune)
 
     def __del__(self):
         if getattr(self, "_h", None):
@@ -146,6 +151,10 @@ class Sentence:
             raise RuntimeError("oracle step refused (max_steps reached)")
         return lse
 
+    def stop_flags(self) -> int:
+        """Bit 0: every hypothesis on the (non-empty) beam is completed; bit 1: some hypothesis is."""
+        return lib().orc_stop_flags(self._h)
+
     def candidates(self):
         cap = self.k * (self.C + 3)
         h = np.zeros(cap, np.int32); w = np.zeros(cap, np.int32); sc = np.zeros(cap, np.float32)
@@ -173,9 +182,9 @@ class Batch:
     sentence is unchanged.
     """
 
-    def __init__(self, k, V, max_steps, constraints, pad=0, bos=1, eos=2, flags=0, threads=1):
+    def __init__(self, k, V, max_steps, constraints, pad=0, bos=1, eos=2, flags=0, threads=1, prune=0.0):
         self.k, self.V, self.B = k, V, len(constraints)
-        self.sent = [Sentence(k, V, max_steps, c, pad, bos, eos, flags) for c in constraints]
+        self.sent = [Sentence(k, V, max_steps, c, pad, bos, eos, flags, prune) for c in constraints]
         self.threads = threads
         self._pool = ThreadPoolExecutor(threads) if threads > 1 else None
 
@@ -189,6 +198,9 @@ class Batch:
     def beam(self):
         bs = [s.beam() for s in self.sent]
         return {key: np.concatenate([b[key] for b in bs]) for key in bs[0]}
+
+    def stop_flags(self):
+        return np.array([s.stop_flags() for s in self.sent], np.int32)
 
     def finalize(self):
         return [s.finalize() for s in self.sent]

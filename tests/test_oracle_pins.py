@@ -429,3 +429,79 @@ def test_row_top_is_a_stable_descending_sort():
             m = min(n, V)
             assert idx[:m].tolist() == order.tolist() and np.array_equal(val[:m], x[order])
             assert (idx[m:] == -1).all() and np.isinf(val[m:]).all()
+
+
+# ------------------------------------------------------------------------------------------ pruning, stopping
+def test_pruning_keeps_exactly_the_hypotheses_within_the_threshold_of_the_best_completed_one():
+    """Section 4: a hypothesis is removed when its log-probability is not within the threshold of the best
+    completed hypothesis.  Vocabulary {pad, bos, eos, a}: the first step offers the end token with logit 0 and
+    `a` with logit -d, so the two continuations score -log(1+e^-d) and -d - log(1+e^-d): exactly d apart."""
+    for d, theta, kept in [(5.0, 20.0, True), (19.5, 20.0, True), (20.5, 20.0, False), (25.0, 20.0, False),
+                           (2.5, 3.0, True), (3.5, 3.0, False), (25.0, 0.0, True)]:
+        s = O.Sentence(3, 4, 2, [], prune=theta)
+        x = np.full((3, 4), NEG, np.float32); x[0, 2] = 0.0; x[0, 3] = -d
+        s.step(x)
+        bm = s.beam()
+        lse = np.log1p(np.exp(-d))
+        assert bm["token"][0] == 2 and abs(bm["score"][0] + lse) < 1e-6
+        if kept:
+            assert bm["token"][1] == 3 and abs(bm["score"][1] + d + lse) < 1e-5 and s.stop_flags() == 2
+        else:       # the slot is empty, and then everything on the beam is completed
+            assert np.isinf(bm["score"][1]) and bm["token"][1] == 0 and bm["bank"][1] == -1 and s.stop_flags() == 3
+        assert np.isinf(bm["score"][2])
+
+
+def test_pruning_removes_completed_hypotheses_too_and_never_the_best_completed_one():
+    k, V = 4, 4
+    s = O.Sentence(k, V, 3, [], prune=20.0)
+    assert s.stop_flags() == 0                       # nothing completed at the start
+    s.set_beam([-1.0, -30.0, -5.0, NEG], [2, 2, 3, 0], [0] * 4, [-1] * 4, [1, 1, 1, 0])
+    x = np.full((k, V), NEG, np.float32); x[2, 2] = 0.0; x[2, 3] = 0.0        # the open one: two equal choices
+    s.step(x)
+    bm = s.beam()
+    half = np.float32(-5.0) + np.float32(-np.log(2.0))
+    assert bm["score"][0] == np.float32(-1.0) and bm["token"][0] == 2 and bm["backptr"][0] == 0
+    assert bm["backptr"][1:3].tolist() == [2, 2] and bm["token"][1:3].tolist() == [2, 3]
+    assert np.allclose(bm["score"][1:3], half, atol=1e-6)
+    assert np.isinf(bm["score"][3])                  # the completed hypothesis at -30 is gone
+    assert s.stop_flags() == 2
+    # without pruning it stays
+    u = O.Sentence(k, V, 3, [])
+    u.set_beam([-1.0, -30.0, -5.0, NEG], [2, 2, 3, 0], [0] * 4, [-1] * 4, [1, 1, 1, 0])
+    u.step(x)
+    assert u.beam()["score"][3] == np.float32(-30.0) and u.beam()["token"][3] == 2
+
+
+def test_stop_bit_zero_needs_every_hypothesis_on_the_beam_completed():
+    s = O.Sentence(3, 5, 4, [])
+    s.set_beam([-1.0, -2.0, NEG], [2, 2, 0], [0] * 3, [-1] * 3, [2, 2, 0])
+    assert s.stop_flags() == 3
+    s.step(np.zeros((3, 5), np.float32))             # completed hypotheses repeat the end token, frozen
+    assert s.stop_flags() == 3 and s.beam()["score"][:2].tolist() == [-1.0, -2.0]
+    s.set_beam([-1.0, -2.0, -3.0], [2, 4, 2], [0] * 3, [-1] * 3, [2, 2, 2])
+    assert s.stop_flags() == 2
+
+
+def test_a_huge_threshold_changes_nothing_and_survivors_are_always_within_the_threshold():
+    rng = np.random.default_rng(5)
+    k, V, T = 6, 40, 14
+    phrases = [[7, 8], [9]]
+    a, b, c = O.Sentence(k, V, T, phrases), O.Sentence(k, V, T, phrases, prune=1e30), O.Sentence(k, V, T, phrases, prune=2.0)
+    pruned_something = False
+    for t in range(T):
+        x = rng.normal(0, 2, (k, V)).astype(np.float32)
+        x[:, 2] += 2.0 if t > 3 else -5.0
+        x[:, 7:10] += 3.0
+        for s in (a, b, c):
+            s.step(x)
+        ba, bb, bc = a.beam(), b.beam(), c.beam()
+        for f in ("score", "token", "backptr", "bank", "met_mask", "active"):
+            assert np.array_equal(ba[f], bb[f])
+        live = np.isfinite(bc["score"])
+        done = live & (bc["token"] == 2)
+        if done.any():
+            best = bc["score"][done].max()
+            assert (bc["score"][live] >= np.float32(best - np.float32(2.0))).all()
+            pruned_something |= live.sum() < np.isfinite(ba["score"]).sum()
+        assert (np.diff(live.astype(int)) <= 0).all()
+    assert pruned_something
