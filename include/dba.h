@@ -53,6 +53,12 @@ enum {
     DBA_FLAG_HOST_STAGING = 4u   /* reserve workspace for dba_step_host                                 */
 };
 
+/* Bits of dba_step_out.stop (Section 4's stopping rule; Section 6.4's early stopping). */
+enum {
+    DBA_STOP_ALL_COMPLETED  = 1,  /* the beam is not empty and every hypothesis on it has generated eos_id */
+    DBA_STOP_SOME_COMPLETED = 2   /* some hypothesis on the beam has generated eos_id                       */
+};
+
 /*
  * Problem statement (Section 3): a fixed beam size k and, per sentence, a set of word constraints (one
  * token) and phrasal constraints (two or more contiguous tokens, met in order).  C_b, the number of
@@ -67,6 +73,9 @@ typedef struct {
     const int32_t* sent_phrase_off;    /* [B+1]  phrases of sentence b are [off[b], off[b+1])             */
     const int32_t* phrase_tok_off;     /* [P+1]  tokens of phrase p are   [off[p], off[p+1]), non-empty   */
     const int32_t* tok;                /* [sum]  token ids in [0, V), none of pad/bos/eos                 */
+    float prune_threshold;             /* Section 4: > 0 removes, after every step, the hypotheses (completed or
+                                          not) whose score is more than this below the best completed
+                                          hypothesis on the beam (the paper uses 20); <= 0: no pruning       */
 } dba_config;
 
 /*
@@ -80,6 +89,10 @@ typedef struct {
  *   met_mask  bit j set = constraint token position j (phrases flattened in order) is marked met
  *   active    position of the last met token of a begun, unfinished phrase, else -1
  *   row_lse   log-sum-exp of the INPUT rows of this step (fp32; 0 for rows that were not open)
+ *   stop      [B], not [B*k]: DBA_STOP_* bits of each sentence's new beam.  The library keeps stepping a
+ *             sentence whatever they say (completed hypotheses repeat eos_id at an unchanged score); the
+ *             caller owns the loop: "all completed" is the paper's stopping rule, "some completed" its
+ *             early-stopping variant.
  */
 typedef struct {
     int32_t*  backptr;
@@ -89,6 +102,7 @@ typedef struct {
     uint64_t* met_mask;
     int32_t*  active;
     float*    row_lse;
+    int32_t*  stop;
 } dba_step_out;
 
 /* Bytes of device workspace a handle for this configuration needs (256-byte aligned base). */
@@ -119,6 +133,8 @@ dba_status dba_reset(dba_handle* h);
  *   Section 3.2      the k slots are divided over the C_b+1 banks (floor(k/(C_b+1)) each, the rest to
  *                    the top bank; unfillable slots move to the nearest banks that can use them) and
  *                    each bank keeps its best candidates.
+ *   Section 4        with prune_threshold > 0, hypotheses of the new beam scoring below (best completed
+ *                    score - prune_threshold) are removed: their slots are empty.
  * row_lse_in_dev (optional, [B*k] fp32): when non-NULL, the row normalisers are taken from it instead
  * of being computed from the logits (e.g. all zeros when the rows are log-probabilities already); the
  * computed values are still what out->row_lse reports.

@@ -29,12 +29,12 @@ class Config(C.Structure):
     _fields_ = [("B", C.c_int32), ("k", C.c_int32), ("V", C.c_int32), ("max_steps", C.c_int32),
                 ("pad_id", C.c_int32), ("bos_id", C.c_int32), ("eos_id", C.c_int32), ("logit_dtype", C.c_int32),
                 ("flags", C.c_uint32), ("sent_phrase_off", C.c_void_p), ("phrase_tok_off", C.c_void_p),
-                ("tok", C.c_void_p)]
+                ("tok", C.c_void_p), ("prune_threshold", C.c_float)]
 
 
 class StepOut(C.Structure):
     _fields_ = [("backptr", C.c_void_p), ("token", C.c_void_p), ("score", C.c_void_p), ("bank", C.c_void_p),
-                ("met_mask", C.c_void_p), ("active", C.c_void_p), ("row_lse", C.c_void_p)]
+                ("met_mask", C.c_void_p), ("active", C.c_void_p), ("row_lse", C.c_void_p), ("stop", C.c_void_p)]
 
 
 _lib = None
@@ -89,10 +89,10 @@ class DbaStepper:
     """Owns a dba_handle and its workspace.  Constraints: per sentence a list of phrases (lists of token ids),
     or the three CSR arrays (sent_phrase_off, phrase_tok_off, tok)."""
 
-    OUT_FIELDS = ("backptr", "token", "score", "bank", "met_mask", "active", "row_lse")
+    OUT_FIELDS = ("backptr", "token", "score", "bank", "met_mask", "active", "row_lse", "stop")
 
     def __init__(self, B, k, V, max_steps, constraints=None, csr=None, dtype=F32, pad=0, bos=1, eos=2, flags=0,
-                 device="cuda:0", stream=None):
+                 device="cuda:0", stream=None, prune=0.0):
         import torch
         self.torch = torch
         self.B, self.k, self.V, self.R, self.max_steps, self.dtype = B, k, V, B * k, max_steps, dtype
@@ -108,7 +108,7 @@ class DbaStepper:
         self._po = np.ascontiguousarray(csr[1], np.int32)
         self._tk = np.ascontiguousarray(csr[2] if len(csr[2]) else [0], np.int32)
         self.cfg = Config(B, k, V, max_steps, pad, bos, eos, dtype, flags, self._so.ctypes.data, self._po.ctypes.data,
-                          self._tk.ctypes.data)
+                          self._tk.ctypes.data, prune)
         n = C.c_size_t()
         _check(lib().dba_workspace_bytes(C.byref(self.cfg), C.byref(n)), "dba_workspace_bytes")
         self.workspace_bytes = n.value
@@ -128,7 +128,8 @@ class DbaStepper:
         return dict(backptr=torch.zeros(R, dtype=torch.int32, **kw), token=torch.zeros(R, dtype=torch.int32, **kw),
                     score=torch.zeros(R, dtype=torch.float32, **kw), bank=torch.zeros(R, dtype=torch.int32, **kw),
                     met_mask=torch.zeros(R, dtype=torch.int64, **kw), active=torch.zeros(R, dtype=torch.int32, **kw),
-                    row_lse=torch.zeros(R, dtype=torch.float32, **kw))
+                    row_lse=torch.zeros(R, dtype=torch.float32, **kw),
+                    stop=torch.zeros(self.B, dtype=torch.int32, **kw))
 
     @staticmethod
     def _out_struct(out):

@@ -127,10 +127,24 @@ allocate_kernel(Dims d, const SentCons* __restrict__ cons, Beam cur, Beam nxt, c
     const Cand* cb = cand + (int64_t)b * d.max_cand;
     for (int i = lane; i < ns; i += 32) { s_score[warp][i] = cb[sel[i]].score; s_flat[warp][i] = cb[sel[i]].flat; }
     __syncwarp();
+    // Section 4: threshold pruning.  Hypotheses scoring below (best completed score - threshold) are removed,
+    // completed or not; they are the tail of the ordered beam, so their slots are simply left empty.
+    float cut = neg_inf();
+    if (d.prune > 0.f) {
+        float best = neg_inf();
+        for (int i = lane; i < ns; i += 32) {
+            const int fi = s_flat[warp][i];
+            if (fi - (fi / V) * V == d.eos_id) best = fmaxf(best, s_score[warp][i]);
+        }
+        best = warp_max(best);
+        if (best != neg_inf()) cut = __fsub_rn(best, d.prune);
+    }
     // new beam in decreasing score order, ties by lower flat index (Section 3.1), empty slots last
     const int r0 = b * k;
+    int n_pruned = 0;
+    for (int i0 = 0; i0 < ns; i0 += 32) n_pruned += __popc(__ballot_sync(kFullMask, i0 + lane < ns && s_score[warp][i0 + lane] < cut));
     for (int i = lane; i < k; i += 32) {
-        if (i < ns) {
+        if (i < ns && !(s_score[warp][i] < cut)) {
             const float si = s_score[warp][i]; const int fi = s_flat[warp][i];
             int rank = 0;
             for (int j = 0; j < ns; ++j) rank += cell_better(s_score[warp][j], s_flat[warp][j], si, fi);
@@ -151,7 +165,7 @@ allocate_kernel(Dims d, const SentCons* __restrict__ cons, Beam cur, Beam nxt, c
             if (out.active) out.active[r] = c.active;
         }
     }
-    for (int i = ns + lane; i < k; i += 32) {
+    for (int i = ns - n_pruned + lane; i < k; i += 32) {
         const int r = r0 + i;
         nxt.score[r] = neg_inf(); nxt.token[r] = d.pad_id; nxt.mask[r] = 0; nxt.active[r] = -1; nxt.len[r] = 0;
         nxt.bank[r] = -1; nxt.backptr[r] = 0;
@@ -167,15 +181,22 @@ allocate_kernel(Dims d, const SentCons* __restrict__ cons, Beam cur, Beam nxt, c
         for (int i = lane; i < k; i += 32) out.row_lse[r0 + i] = row_lse[r0 + i];
     // rows the next step has to scan: live slots that have not generated the end token
     __syncwarp();
+    int n_live = 0, n_done = 0;
     for (int i0 = 0; i0 < k; i0 += 32) {
         const int i = i0 + lane;
-        const bool open = i < k && nxt.score[r0 + i] != neg_inf() && nxt.token[r0 + i] != d.eos_id;
+        const bool live = i < k && nxt.score[r0 + i] != neg_inf();
+        const bool open = live && nxt.token[r0 + i] != d.eos_id;
+        n_live += __popc(__ballot_sync(kFullMask, live));
+        n_done += __popc(__ballot_sync(kFullMask, live && !open));
         const unsigned bal = __ballot_sync(kFullMask, open);
         int base = 0;
         if (lane == 0 && bal) base = atomicAdd(open_count, __popc(bal));
         base = __shfl_sync(kFullMask, base, 0);
         if (open) open_list[base + __popc(bal & ((1u << lane) - 1u))] = r0 + i;
     }
+    // Section 4's stopping rule (everything on the beam completed) and Section 6.4's early stopping (something is)
+    if (out.stop && lane == 0)
+        out.stop[b] = (n_live > 0 && n_done == n_live ? DBA_STOP_ALL_COMPLETED : 0) | (n_done > 0 ? DBA_STOP_SOME_COMPLETED : 0);
 }
 
 // Algorithm 1, DECODER-INIT: slot 0 holds the start symbol at score 0, the other slots are empty.

@@ -66,6 +66,7 @@ dba_status check_config(const dba_config* c, Shape* shape, std::vector<SentCons>
     if (!c) return DBA_ERR_INVALID_ARG;
     if (c->B < 1 || c->k < 1 || c->V < 1 || c->max_steps < 1) return DBA_ERR_INVALID_ARG;
     if (c->logit_dtype != DBA_F32 && c->logit_dtype != DBA_BF16) return DBA_ERR_INVALID_ARG;
+    if (c->prune_threshold != c->prune_threshold) return DBA_ERR_INVALID_ARG;      // NaN
     if (c->flags & ~(DBA_FLAG_ADJUST_OFF | DBA_FLAG_LENGTH_NORM | DBA_FLAG_HOST_STAGING)) return DBA_ERR_INVALID_ARG;
     const int32_t sp[3] = {c->pad_id, c->bos_id, c->eos_id};
     for (int i = 0; i < 3; ++i)
@@ -116,6 +117,7 @@ void fill_dims(const dba_config* c, const Shape& sh, Dims* d) {
     d->B = c->B; d->k = c->k; d->V = c->V; d->R = c->B * c->k;
     d->pad_id = c->pad_id; d->bos_id = c->bos_id; d->eos_id = c->eos_id;
     d->dtype = c->logit_dtype; d->flags = c->flags;
+    d->prune = c->prune_threshold > 0.f ? c->prune_threshold : 0.f;
     d->max_cand = c->k * (sh.max_phrases + 2);
     d->K1 = c->k + 2; d->S = kMaxSeg; d->seg_len = 0;   // S is an upper bound until plan_segments runs
 }
@@ -161,6 +163,7 @@ size_t carve(dba_handle* h, void* base, int32_t max_steps) {
         h->stage_out.score = cv.take<float>(R); h->stage_out.bank = cv.take<int32_t>(R);
         h->stage_out.met_mask = cv.take<uint64_t>(R); h->stage_out.active = cv.take<int32_t>(R);
         h->stage_out.row_lse = cv.take<float>(R);
+        h->stage_out.stop = cv.take<int32_t>(d.B);
     }
     return (cv.off + 255) / 256 * 256;
 }
@@ -299,6 +302,7 @@ dba_status dba_step_host(dba_handle* h, const void* logits_host, int64_t row_str
         if (out_host->met_mask && e == cudaSuccess) e = cudaMemcpyAsync(out_host->met_mask, s.met_mask, R * 8, k, h->stream);
         if (out_host->active && e == cudaSuccess) e = cudaMemcpyAsync(out_host->active, s.active, R * 4, k, h->stream);
         if (out_host->row_lse && e == cudaSuccess) e = cudaMemcpyAsync(out_host->row_lse, s.row_lse, R * 4, k, h->stream);
+        if (out_host->stop && e == cudaSuccess) e = cudaMemcpyAsync(out_host->stop, s.stop, (size_t)h->d.B * 4, k, h->stream);
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
     return cuda_fail(e);

@@ -59,6 +59,7 @@ struct Dims {
     int32_t pad_id, bos_id, eos_id;
     int32_t dtype;
     uint32_t flags;
+    float prune;       // Section 4's pruning threshold (<= 0: off)
 };
 
 // Partial results of the row scan, one entry per (row, segment).

@@ -32,6 +32,8 @@ def to_host_logits(x_dev):
 def gpu_beam(out):
     d = {f: out[f].cpu().numpy() for f in ("backptr", "token", "score", "bank", "active", "row_lse")}
     d["met_mask"] = out["met_mask"].cpu().numpy().view(np.uint64)
+    if out.get("stop") is not None:
+        d["stop"] = out["stop"].cpu().numpy()
     return d
 
 
@@ -49,13 +51,13 @@ def assert_beam_equal(got, want, where, fields=BEAM_FIELDS + ("score",)):
                                  f"gpu    {({g: got[g][r] for g in fields})}\noracle {({g: want[g][r] for g in fields})}")
 
 
-def lockstep(wl, stepper, steps=None, threads=8, gpu_gen=None, lse_tol=1e-5, flags=0):
+def lockstep(wl, stepper, steps=None, threads=8, gpu_gen=None, lse_tol=1e-5, flags=0, prune=0.0):
     """Closed loop with the oracle's row normalisers handed to the CUDA step (the direction oracle -> GPU),
     so that both rank the same fp32 score matrix: every selection output must then match bit for bit at
     every step, and the normalisers the GPU computes itself must agree within lse_tol."""
     import torch
     steps = wl.steps if steps is None else steps
-    orc = O.Batch(wl.k, wl.V, steps, wl.constraints, flags=flags & 3, threads=threads)
+    orc = O.Batch(wl.k, wl.V, steps, wl.constraints, flags=flags & 3, threads=threads, prune=prune)
     host_gen = LogitStream(wl) if gpu_gen is None else None
     worst = 0.0
     for t in range(steps):
@@ -72,6 +74,7 @@ def lockstep(wl, stepper, steps=None, threads=8, gpu_gen=None, lse_tol=1e-5, fla
         out = stepper.step(x_dev, row_lse_in=torch.from_numpy(lse_o).cuda())
         g = gpu_beam(out)
         assert_beam_equal(g, orc.beam(), f"{wl.name} step {t}")
+        assert np.array_equal(g["stop"], orc.stop_flags()), f"{wl.name} step {t}: stop bits differ"
         err = np.abs(g["row_lse"][open_rows].astype(np.float64) - lse_o[open_rows]).max() if open_rows.any() else 0.0
         worst = max(worst, float(err))
         assert err <= lse_tol, f"{wl.name} step {t}: row normaliser off by {err}"

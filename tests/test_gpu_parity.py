@@ -180,6 +180,20 @@ def test_step_parity_edge_cases(dba, case):
     assert_finalize_equal(st, orc)
 
 
+@pytest.mark.parametrize("name,kw,theta", [("tiny", {}, 3.0), ("ragged", dict(B=6, V=4096, steps=40), 20.0),
+                                           ("ragged", dict(B=6, V=4096, steps=40), 2.0),
+                                           ("serving", dict(B=3, V=8192, steps=60), 5.0)])
+def test_threshold_pruning_and_stop_bits_match_the_oracle(dba, name, kw, theta):
+    wl = make_workload(name, **kw)
+    st = dba.DbaStepper(wl.B, wl.k, wl.V, wl.steps, constraints=wl.constraints,
+                        dtype=dba.BF16 if wl.dtype == "bf16" else dba.F32, prune=theta)
+    orc, worst = lockstep(wl, st, prune=theta)
+    assert_finalize_equal(st, orc)
+    flags = orc.stop_flags()
+    assert name == "tiny" or (flags & 2).any()      # the stream does complete hypotheses: the pruning had work to do
+    st.close()
+
+
 @pytest.mark.parametrize("flags", [1, 2, 3])
 def test_flags_adjust_off_and_length_norm(dba, flags):
     wl = make_workload("ragged", B=6, V=3000, steps=50)
