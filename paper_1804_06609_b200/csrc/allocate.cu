@@ -36,6 +36,8 @@ allocate_kernel(Dims d, const SentCons* __restrict__ cons, Beam cur, Beam nxt, c
     __shared__ int s_flat[kAllocWarps][kMaxK];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x * kAllocWarps + warp;
+    if (threadIdx.x == 0) allow_dependents();
+    grid_dependency_wait();      // the candidates come from the kernel before
     if (b >= d.B) return;
     const int k = d.k, V = d.V;
     const int C = cons[b].C;
@@ -261,10 +263,9 @@ cudaError_t launch_allocate(const Dims& d, const SentCons* cons, const Beam& cur
                             const Cand* cand, const int32_t* ncand, const int32_t* bank_count,
                             const float* row_lse, const dba_step_out& out, int32_t* hist_bp, int32_t* hist_tok,
                             int32_t* open_list, int32_t* open_count, cudaStream_t st, int* launches) {
-    allocate_kernel<<<(d.B + kAllocWarps - 1) / kAllocWarps, kAllocWarps * 32, 0, st>>>(
-        d, cons, cur, next, cand, ncand, bank_count, row_lse, out, hist_bp, hist_tok, open_list, open_count);
     ++*launches;
-    return cudaGetLastError();
+    return launch_after(allocate_kernel, dim3((d.B + kAllocWarps - 1) / kAllocWarps), dim3(kAllocWarps * 32), 0, st,
+                        d, cons, cur, next, cand, ncand, bank_count, row_lse, out, hist_bp, hist_tok, open_list, open_count);
 }
 
 cudaError_t launch_reset(const Dims& d, const Beam& beam, int32_t* open_list, int32_t* open_count,

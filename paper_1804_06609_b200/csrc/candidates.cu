@@ -95,6 +95,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r0 = b * k;
+    if (tid == 0) allow_dependents();
 
     // ---- load the sentence: constraint table and beam state --------------------------------------------
     {
@@ -114,6 +115,9 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     }
     if (tid <= kMaxC) bank_cnt[tid] = 0;
     if (tid == 0) { s_ncand = 0; s_ns1 = 0; }
+    // Up to here only what earlier steps left behind was read (the row scan waited for them before it let
+    // this kernel start); from here on the row scan's own results are needed.
+    grid_dependency_wait();
     if (tid == 0 && blockIdx.x == 0) *open_count = 0;   // the allocation kernel rebuilds the list of open rows
     __syncthreads();
     const int C = sc.C;
@@ -533,10 +537,9 @@ cudaError_t launch_candidates(const void* logits, int64_t stride, const Dims& d,
                               int32_t* open_count, cudaStream_t st, int* launches) {
     const int threads = pick_threads(d, g_smem_limit);
     const size_t smem = (size_t)make_layout(d.k, d.K1, d.S, d.max_cand, threads / 32).total;
-    candidates_kernel<<<d.B, threads, smem, st>>>(logits, stride, d, cons, cur, part, lse_in, row_lse, cand,
-                                                  ncand, bank_count, status, open_count);
     ++*launches;
-    return cudaGetLastError();
+    return launch_after(candidates_kernel, dim3(d.B), dim3(threads), smem, st, logits, stride, d, cons, cur, part, lse_in,
+                        row_lse, cand, ncand, bank_count, status, open_count);
 }
 
 }  // namespace dba

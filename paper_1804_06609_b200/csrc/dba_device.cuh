@@ -8,6 +8,14 @@ namespace dba {
 
 constexpr unsigned kFullMask = 0xffffffffu;
 
+// Programmatic dependent launch: the three kernels of a step follow one another on a stream.  A kernel
+// launched with launch_after() may start while its predecessor is still running; it must not touch what the
+// predecessor produces (or still reads and this kernel writes) before grid_dependency_wait() returns, which
+// is when the predecessor has finished and its writes are visible.  allow_dependents() lets the successor's
+// blocks be scheduled as soon as there is room for them.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void allow_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 
 // Monotone map float -> uint32 (larger float, larger integer).  -0.0 is folded onto +0.0 first so that

@@ -70,6 +70,20 @@ struct ScanOut {
     int32_t* top_idx;  // [R*S*K1] column within the row
 };
 
+// Launch with programmatic stream serialisation: the kernel may begin before the previous kernel of the
+// stream has finished (see grid_dependency_wait in dba_device.cuh).
+template <typename... Params, typename... Args>
+inline cudaError_t launch_after(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 // --- launchers (each enqueues on `st` and returns the CUDA error of the launch) ----------------------
 // `open_score` / `open_token` (may be null): rows whose slot is empty (score -inf) or finished
 // (token == eos) are skipped.

@@ -308,6 +308,8 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    grid_dependency_wait();      // the list of open rows comes from the previous step's last kernel
+    if (tid == 0) allow_dependents();
 
     if (warp == kWarpProd) {
         // ------------------------------------------------------------------ producer
@@ -660,9 +662,8 @@ cudaError_t launch_row_scan_tma(const void* logits, int64_t stride, const Dims& 
     p.part_m = out.m; p.part_s = out.s; p.top_val = out.top_val; p.top_idx = out.top_idx; p.status = status;
     const int64_t items = (int64_t)d.R * d.S;
     const int grid = (int)(items < sm_count ? items : sm_count);
-    if (d.dtype == DBA_F32) row_scan_tma_kernel<float><<<grid, kThreads, row_scan_tma_smem(), st>>>(p);
-    else row_scan_tma_kernel<__nv_bfloat16><<<grid, kThreads, row_scan_tma_smem(), st>>>(p);
-    return cudaGetLastError();
+    if (d.dtype == DBA_F32) return launch_after(row_scan_tma_kernel<float>, dim3(grid), dim3(kThreads), row_scan_tma_smem(), st, p);
+    return launch_after(row_scan_tma_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), row_scan_tma_smem(), st, p);
 }
 
 }  // namespace dba
