@@ -62,7 +62,23 @@ __host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand
     return L;
 }
 
-__global__ void __launch_bounds__(kCandMaxThreads)
+// Merge of descending key lists of at most 32 entries each (key 0 = empty), one entry per lane: with the second
+// list reversed, the lane-wise maximum holds the 32 largest of both as a bitonic sequence, which five
+// compare-exchange steps put in descending order.
+__device__ __forceinline__ uint64_t merge_top32(uint64_t a, uint64_t b, int lane) {
+    const uint64_t br = __shfl_sync(kFullMask, b, 31 - lane);
+    uint64_t acc = a > br ? a : br;
+#pragma unroll
+    for (int str = 16; str; str >>= 1) {
+        const uint64_t o = __shfl_xor_sync(kFullMask, acc, str);
+        const bool upper = (lane & str) == 0;             // this lane keeps the larger of the pair
+        acc = (o > acc) == upper ? o : acc;
+    }
+    return acc;
+}
+
+// 48 registers: two CTAs of 640 threads (a warp per row at k = 20) fit an SM.
+__global__ void __maxnreg__(48)
 candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const SentCons* __restrict__ cons,
                   Beam cur, ScanOut part, const float* __restrict__ lse_in, float* __restrict__ row_lse,
                   Cand* __restrict__ cand_out, int32_t* __restrict__ ncand_out, int32_t* __restrict__ bank_count,
@@ -168,6 +184,11 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
             const int n = n_ent;
             for (int e = lane; e < K1; e += 32) merged[e] = 0ull;
             __syncwarp();
+            if (K1 <= 32) {
+                uint64_t acc = lane < K1 ? stage[lane] : 0ull;
+                for (int g = 1; g < S; ++g) acc = merge_top32(acc, lane < K1 ? stage[g * K1 + lane] : 0ull, lane);
+                if (lane < K1) merged[lane] = acc;
+            } else
             // every segment's list is in descending key order (empty entries, key 0, last): the place of an
             // entry in the merged order is its place in its own list plus, for every other list, the number of
             // keys above it, found by bisection
@@ -506,12 +527,14 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
 
 }  // namespace
 
-// Threads per CTA: 1024 when every sentence gets an SM of its own (then only the latency of one CTA counts),
-// 512 otherwise (two CTAs fit an SM's registers); fewer if the per-warp scratch would not fit shared memory.
+// Threads per CTA: 1024 when every sentence gets an SM of its own (then only the latency of one CTA counts);
+// otherwise two CTAs share an SM: 640 threads when the beam has more than 16 rows (a warp per row up to k = 20),
+// else 512; fewer if the per-warp scratch would not fit shared memory.
 static size_t g_smem_limit = 48 * 1024;     // raised by configure_candidates
 static int g_sm_count = 1;
 static int pick_threads(const Dims& d, size_t smem_limit) {
-    for (int t = d.B <= g_sm_count ? kCandMaxThreads : kCandMaxThreads / 2; t > 256; t >>= 1)
+    const int first = d.B <= g_sm_count ? kCandMaxThreads : (d.k > 16 ? 640 : 512);
+    for (int t = first; t > 256; t = t == 640 ? 512 : t >> 1)
         if ((size_t)make_layout(d.k, d.K1, d.S, d.max_cand, t / 32).total <= smem_limit) return t;
     return 256;
 }
