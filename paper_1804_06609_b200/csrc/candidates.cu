@@ -19,7 +19,7 @@ struct SortEnt {
 };
 
 struct Layout {   // byte offsets into dynamic shared memory
-    int cons, parent, lse, mask, active, kind, eos_ok, rt_score, rt_w, rt_n, rt_ptr, s1_h, s1_i, stage, merged,
+    int cons, parent, lse, mask, active, kind, eos_ok, s2_x, rt_score, rt_w, rt_n, rt_ptr, s1_h, s1_i, stage, merged,
         tmp_score, tmp_w, tmp_x, c_score, c_flat, c_mask, c_active, bank_cnt, sort, total;
     int n_sort;
 };
@@ -37,6 +37,7 @@ __host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand
     L.active = o;    o += 4 * k;
     L.kind = o;      o += 4 * k;
     L.eos_ok = o;    o += 4 * k;
+    L.s2_x = o;      o += 4 * k * kMaxC;
     L.rt_score = o;  o += 4 * k * k;
     L.rt_w = o;      o += 4 * k * k;
     L.rt_n = o;      o += 4 * k;
@@ -77,7 +78,7 @@ __device__ __forceinline__ uint64_t merge_top32(uint64_t a, uint64_t b, int lane
     return acc;
 }
 
-// 48 registers: two CTAs of 640 threads (a warp per row at k = 20) fit an SM.
+// 48 registers: two CTAs of 672 threads (a warp per row at k = 20, and one more) fit an SM.
 __global__ void __maxnreg__(48)
 candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const SentCons* __restrict__ cons,
                   Beam cur, ScanOut part, const float* __restrict__ lse_in, float* __restrict__ row_lse,
@@ -94,6 +95,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     int* s_active = reinterpret_cast<int*>(smem + L.active);
     int* s_kind = reinterpret_cast<int*>(smem + L.kind);      // 0 empty, 1 open, 2 finished
     int* s_eos_ok = reinterpret_cast<int*>(smem + L.eos_ok);
+    float* s2_x = reinterpret_cast<float*>(smem + L.s2_x);    // logit of the token at constraint position j of row h, if it advances h
     float* rt_score = reinterpret_cast<float*>(smem + L.rt_score);
     int* rt_w = reinterpret_cast<int*>(smem + L.rt_w);
     int* rt_n = reinterpret_cast<int*>(smem + L.rt_n);
@@ -131,6 +133,32 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     }
     if (tid <= kMaxC) bank_cnt[tid] = 0;
     if (tid == 0) { s_ncand = 0; s_ns1 = 0; }
+    // Source 2's logits, fetched early: which tokens advance a hypothesis depends on the beam alone, and the
+    // logits were there before the row scan started.  These are scattered reads of a matrix that has left the
+    // L2 cache, the longest single latency of this kernel; here it overlaps the end of the row scan.
+    __syncthreads();
+    {
+        const int C0 = sc.C;
+        for (int h = warp; h < k; h += n_warps) {
+            if (s_kind[h] != 1) continue;
+            const uint64_t m = s_mask[h]; const int a = s_active[h];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int j = lane + 32 * q;
+                bool ok = j < C0;
+                if (ok) {
+                    if (a >= 0) ok = j == a + 1;
+                    else {
+                        ok = ((sc.first_mask >> j) & 1ull) && !((m >> j) & 1ull);
+                        // the same token may open an earlier word/phrase that is still unmet: then that one is listed
+                        for (int e = ok ? sc.prev_same[j] : 255; e != 255; e = sc.prev_same[e])
+                            if (!((m >> e) & 1ull)) { ok = false; break; }
+                    }
+                }
+                s2_x[h * kMaxC + j] = ok ? load_logit_dyn(logits, d.dtype, (int64_t)(r0 + h) * stride + sc.ctok[j]) : neg_inf();
+            }
+        }
+    }
     // Up to here only what earlier steps left behind was read (the row scan waited for them before it let
     // this kernel start); from here on the row scan's own results are needed.
     grid_dependency_wait();
@@ -334,26 +362,15 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         //      counts at least k candidates, which is all the allocation needs to know).
         for (int h = warp - 1; h < k; h += n_warps - 1) {
             if (s_kind[h] != 1) continue;
-            const uint64_t m = s_mask[h]; const int a = s_active[h];
+            const uint64_t m = s_mask[h];
             const float lse = s_lse[h], parent = s_parent[h];
             float sc2[2]; int w2[2], j2[2]; bool v2[2];
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 const int j = lane + 32 * q;
-                bool ok = j < C && lse != neg_inf();
-                if (ok) {
-                    if (a >= 0) ok = j == a + 1;
-                    else {
-                        ok = ((sc.first_mask >> j) & 1ull) && !((m >> j) & 1ull);
-                        // the same token may open an earlier word/phrase that is still unmet: then that one is listed
-                        for (int e = ok ? sc.prev_same[j] : 255; e != 255; e = sc.prev_same[e])
-                            if (!((m >> e) & 1ull)) { ok = false; break; }
-                    }
-                }
-                float x = neg_inf();
-                if (ok) { w2[q] = sc.ctok[j]; x = load_logit_dyn(logits, d.dtype, (int64_t)(r0 + h) * stride + w2[q]); }
-                else w2[q] = 0x7fffffff;
-                v2[q] = ok && x != neg_inf();
+                const float x = s2_x[h * kMaxC + j];          // -inf unless the token at position j advances h
+                v2[q] = j < C && lse != neg_inf() && x != neg_inf();
+                w2[q] = v2[q] ? sc.ctok[j] : 0x7fffffff;
                 sc2[q] = v2[q] ? cell_score(x, lse, parent) : neg_inf();
                 j2[q] = j;
             }
@@ -528,12 +545,12 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
 }  // namespace
 
 // Threads per CTA: 1024 when every sentence gets an SM of its own (then only the latency of one CTA counts);
-// otherwise two CTAs share an SM: 640 threads when the beam has more than 16 rows (a warp per row up to k = 20),
-// else 512; fewer if the per-warp scratch would not fit shared memory.
+// otherwise two CTAs share an SM: 672 threads when the beam has more than 15 rows (a warp per row up to k = 20
+// beside the warp that runs the tournament), else 512; fewer if the per-warp scratch would not fit shared memory.
 static size_t g_smem_limit = 48 * 1024;     // raised by configure_candidates
 static int g_sm_count = 1;
 static int pick_threads(const Dims& d, size_t smem_limit) {
-    const int first = d.B <= g_sm_count ? kCandMaxThreads : (d.k > 16 ? 640 : 512);
+    const int first = d.B <= g_sm_count ? kCandMaxThreads : (d.k > 15 ? 640 : 512);
     for (int t = first; t > 256; t = t == 640 ? 512 : t >> 1)
         if ((size_t)make_layout(d.k, d.K1, d.S, d.max_cand, t / 32).total <= smem_limit) return t;
     return 256;
