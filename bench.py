@@ -3,7 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
-A step is one dba_step call: all three kernels over one batch of logits.  The logit stream is generated
+A step is one dba_step call: both kernels (row scan; candidates + allocation) over one batch of logits.  The logit stream is generated
 once, untimed, by running the step in closed loop (every row depends on the hypothesis' last token), and
 kept resident in HBM; the timed loop then replays it, resetting the beam whenever the stream wraps.
 One JSON line is printed by rank 0.  With N > 1 every rank runs an independent replica (sentences do not
@@ -293,7 +293,7 @@ def run_ours(args):
                          if step_bytes > L2_BYTES else f"{T} rotating step buffers, {T * step_bytes >> 20} MiB in all",
                    "parallelism": "replicas" if world > 1 else "single GPU"},
         "hyp_steps_per_sec": value * wl.R,
-        "kernel_ms": {"row_scan": scan_ms, "candidates": kt[1] / ksteps, "allocate": kt[2] / ksteps},
+        "kernel_ms": {"row_scan": scan_ms, "candidates_and_allocation": kt[1] / ksteps},
         "roofline": {"bound": "hbm", "kernel": "row_scan", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs_nominal": achieved / 8000.0,
                      "algorithmic_bytes_per_launch": kbytes / ksteps, "traffic": traffic},

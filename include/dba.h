@@ -164,10 +164,11 @@ dba_status dba_finalize(dba_handle* h, int32_t* tokens_host, int32_t* len_host, 
                         int32_t* flags_host);
 
 /*
- * Optional per-kernel timing for benchmarks.  While enabled, dba_step brackets each of its three kernels
- * (row scan; candidates; allocation) with CUDA events on the handle's stream.  dba_timing_read waits for
- * the stream, adds up the elapsed milliseconds of every step recorded since the last read into
- * ms_total[0..2], stores the number of steps in *steps and clears the record.  At most 4096 steps are
+ * Optional per-kernel timing for benchmarks.  While enabled, dba_step brackets each of its two kernels
+ * (row scan; candidates with the allocation at their end) with CUDA events on the handle's stream.
+ * dba_timing_read waits for the stream, adds up the elapsed milliseconds of every step recorded since the last
+ * read into ms_total[0..1] (ms_total[2] is 0: the allocation has no kernel of its own), stores the number of
+ * steps in *steps and clears the record.  At most 4096 steps are
  * kept between reads (further steps are not recorded).  Off by default.
  */
 dba_status dba_timing_enable(dba_handle* h, int32_t on);

@@ -170,7 +170,7 @@ class DbaStepper:
         _check(lib().dba_timing_enable(self._h, int(on)), "dba_timing_enable")
 
     def timing_read(self):
-        """(ms of [row scan, candidates, allocation] summed over the recorded steps, number of steps)."""
+        """(ms of [row scan, candidates + allocation, 0] summed over the recorded steps, number of steps)."""
         ms = (C.c_double * 3)(); n = C.c_int64()
         _check(lib().dba_timing_read(self._h, ms, C.byref(n)), "dba_timing_read")
         return list(ms), n.value

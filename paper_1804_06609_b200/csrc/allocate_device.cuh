@@ -1,0 +1,215 @@
+// Allocation (Section 3.2: ALLOCATE of Algorithm 2, then newBeam; Section 4's pruning and stopping rule), the
+// last part of a step: one warp per sentence, called by the candidate kernel once the sentence's candidates,
+// grouped by bank and ordered inside each bank, are in shared memory.
+#pragma once
+#include "dba_device.cuh"
+#include "dba_internal.h"
+
+namespace dba {
+
+constexpr int kBanks = kMaxC + 1;
+
+// Nearest bank above / below b whose bit is set in the 65-bit set (lo: banks 0..63, hi: bank 64); -1 if none.
+__device__ __forceinline__ int next_above(uint64_t lo, bool hi, int b) {
+    if (b < 63) {
+        const uint64_t m = lo & ~((2ull << b) - 1ull);
+        if (m) return __ffsll((long long)m) - 1;
+    }
+    return (hi && b < 64) ? 64 : -1;
+}
+__device__ __forceinline__ int next_below(uint64_t lo, int b) {
+    const uint64_t m = b >= 64 ? lo : (lo & ((1ull << b) - 1ull));
+    return m ? 63 - __clzll((long long)m) : -1;
+}
+
+// What the allocation reads of the candidate kernel's shared memory.
+struct AllocIn {
+    const int* bank_cnt;       // [C + 1] candidates per bank
+    const int* order;          // [n] candidate ids in (bank asc, score desc, flat index asc) order
+    const float* c_score;      // by candidate id
+    const int* c_flat;
+    const uint64_t* c_mask;
+    const int* c_active;
+    const int* par_kind;       // [k] of the current beam: 0 empty, 1 open, 2 finished
+    const int* par_len;        // [k] generated tokens so far
+};
+
+// One warp.  Writes the sentence's new beam (and the requested outputs, the history, the stop bits) and appends
+// its open rows to the list the next step's row scan reads.
+__device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, const AllocIn& in, const Beam& nxt,
+                                                  const float* __restrict__ row_lse, const dba_step_out& out,
+                                                  int32_t* __restrict__ hist_bp, int32_t* __restrict__ hist_tok,
+                                                  int32_t* __restrict__ open_list, int32_t* __restrict__ open_count) {
+    __shared__ int n[kBanks];
+    __shared__ int alloc[kBanks];
+    __shared__ int off[kBanks];
+    __shared__ int sel[kMaxK];
+    __shared__ float a_score[kMaxK];
+    __shared__ int a_flat[kMaxK];
+    __shared__ int a_tok[kMaxK];
+    const int lane = threadIdx.x & 31;
+    const int k = d.k, V = d.V;
+    const int* bank_cnt = in.bank_cnt; const int* order = in.order;
+    const float* c_score = in.c_score; const int* c_flat = in.c_flat;
+    const uint64_t* c_mask = in.c_mask; const int* c_active = in.c_active;
+    const int* par_kind = in.par_kind; const int* par_len = in.par_len;
+
+    // Lane l looks after banks l, l + 32 and l + 64 (there are at most 65).
+    // bank sizes; equal base share, remainder to the top bank C (Section 3.2); offsets of the banks inside the
+    // bank-ordered candidate list
+    const int share = k / (C + 1);
+    int nq[3], aq[3];
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+        const int q = lane + 32 * j;
+        nq[j] = q <= C ? bank_cnt[q] : 0;
+        aq[j] = q <= C ? share + (q == C ? k - share * (C + 1) : 0) : 0;
+    }
+    {
+        int run = 0;                                  // exclusive prefix of n over banks, 32 at a time
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+            int incl = nq[j];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(kFullMask, incl, o); if (lane >= o) incl += t; }
+            const int q = lane + 32 * j;
+            if (q <= C) { off[q] = run + incl - nq[j]; n[q] = nq[j]; }
+            run += __shfl_sync(kFullMask, incl, 31);
+        }
+    }
+    if (d.flags & DBA_FLAG_ADJUST_OFF) {
+#pragma unroll
+        for (int j = 0; j < 3; ++j) { const int q = lane + 32 * j; if (q <= C) alloc[q] = min(aq[j], nq[j]); }
+        __syncwarp();
+    } else {
+        // Adjustment: every bank with more slots than candidates passes the surplus to the nearest banks that
+        // have more candidates than slots, the higher one first at equal distance.  The sets of such banks are
+        // bit masks (banks 0..63 in a 64-bit word, bank 64 apart); the walk itself is short and serial.
+        const unsigned o0 = __ballot_sync(kFullMask, aq[0] > nq[0]), o1 = __ballot_sync(kFullMask, aq[1] > nq[1]);
+        const unsigned d0 = __ballot_sync(kFullMask, nq[0] > aq[0]), d1 = __ballot_sync(kFullMask, nq[1] > aq[1]);
+        const bool over_hi = __any_sync(kFullMask, lane == 0 && aq[2] > nq[2]);
+        bool need_hi = __any_sync(kFullMask, lane == 0 && nq[2] > aq[2]);
+        const uint64_t over_lo = (uint64_t)o0 | ((uint64_t)o1 << 32);
+        uint64_t need_lo = (uint64_t)d0 | ((uint64_t)d1 << 32);
+#pragma unroll
+        for (int j = 0; j < 3; ++j) { const int q = lane + 32 * j; if (q <= C) alloc[q] = aq[j]; }
+        __syncwarp();
+        if (lane == 0) {
+            uint64_t todo = over_lo;
+            bool todo_hi = over_hi;
+            while (todo || todo_hi) {
+                int q;
+                if (todo) { q = __ffsll((long long)todo) - 1; todo &= todo - 1; } else { q = 64; todo_hi = false; }
+                int surplus = alloc[q] - n[q];
+                alloc[q] = n[q];
+                while (surplus > 0) {
+                    const int up = next_above(need_lo, need_hi, q);
+                    const int dn = next_below(need_lo, q);
+                    int r;
+                    if (up < 0 && dn < 0) break;
+                    if (up >= 0 && (dn < 0 || up - q <= q - dn)) r = up; else r = dn;
+                    const int g = min(surplus, n[r] - alloc[r]);
+                    alloc[r] += g; surplus -= g;
+                    if (alloc[r] == n[r]) { if (r < 64) need_lo &= ~(1ull << r); else need_hi = false; }
+                }
+            }
+        }
+        __syncwarp();
+    }
+    // the best alloc[q] candidates of every bank (they are ordered inside the bank already)
+    int ns_total;
+    {
+        int run = 0;
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+            const int q = lane + 32 * j;
+            const int a = q <= C ? alloc[q] : 0;
+            int incl = a;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(kFullMask, incl, o); if (lane >= o) incl += t; }
+            const int first = run + incl - a;
+            for (int i = 0; i < a; ++i) sel[first + i] = off[q] + i;
+            run += __shfl_sync(kFullMask, incl, 31);
+        }
+        ns_total = run;
+    }
+    __syncwarp();
+    if (lane == 0) off[0] = ns_total;   // (kept where the code below reads it)
+    __syncwarp();
+    const int ns = off[0];
+    for (int i = lane; i < ns; i += 32) { const int id = order[sel[i]]; sel[i] = id; a_score[i] = c_score[id]; a_flat[i] = c_flat[id]; }
+    __syncwarp();
+    // Section 4: threshold pruning.  Hypotheses scoring below (best completed score - threshold) are removed,
+    // completed or not; they are the tail of the ordered beam, so their slots are simply left empty.
+    float cut = neg_inf();
+    if (d.prune > 0.f) {
+        float best = neg_inf();
+        for (int i = lane; i < ns; i += 32) {
+            const int fi = a_flat[i];
+            if (fi - (fi / V) * V == d.eos_id) best = fmaxf(best, a_score[i]);
+        }
+        best = warp_max(best);
+        if (best != neg_inf()) cut = __fsub_rn(best, d.prune);
+    }
+    // new beam in decreasing score order, ties by lower flat index (Section 3.1), empty slots last
+    const int r0 = b * k;
+    int n_pruned = 0;
+    for (int i0 = 0; i0 < ns; i0 += 32) n_pruned += __popc(__ballot_sync(kFullMask, i0 + lane < ns && a_score[i0 + lane] < cut));
+    for (int i = lane; i < k; i += 32) {
+        if (i < ns && !(a_score[i] < cut)) {
+            const float si = a_score[i]; const int fi = a_flat[i];
+            int rank = 0;
+            for (int j = 0; j < ns; ++j) rank += cell_better(a_score[j], a_flat[j], si, fi);
+            const int id = sel[i];
+            const uint64_t cmask = c_mask[id]; const int cactive = c_active[id];
+            const int h = fi / V, w = fi - h * V;
+            const int r = r0 + rank;
+            const int bank = __popcll(cmask);
+            const int len = par_kind[h] == 2 ? par_len[h] : par_len[h] + 1;      // a finished hypothesis stays as long as it was
+            nxt.score[r] = si; nxt.token[r] = w; nxt.mask[r] = cmask; nxt.active[r] = cactive; nxt.len[r] = len;
+            nxt.bank[r] = bank; nxt.backptr[r] = h;
+            a_tok[rank] = w;
+            hist_bp[r] = h; hist_tok[r] = w;
+            if (out.backptr) out.backptr[r] = h;
+            if (out.token) out.token[r] = w;
+            if (out.score) out.score[r] = si;
+            if (out.bank) out.bank[r] = bank;
+            if (out.met_mask) out.met_mask[r] = cmask;
+            if (out.active) out.active[r] = cactive;
+        }
+    }
+    for (int i = ns - n_pruned + lane; i < k; i += 32) {
+        const int r = r0 + i;
+        nxt.score[r] = neg_inf(); nxt.token[r] = d.pad_id; nxt.mask[r] = 0; nxt.active[r] = -1; nxt.len[r] = 0;
+        nxt.bank[r] = -1; nxt.backptr[r] = 0;
+        hist_bp[r] = 0; hist_tok[r] = d.pad_id;
+        if (out.backptr) out.backptr[r] = 0;
+        if (out.token) out.token[r] = d.pad_id;
+        if (out.score) out.score[r] = neg_inf();
+        if (out.bank) out.bank[r] = -1;
+        if (out.met_mask) out.met_mask[r] = 0;
+        if (out.active) out.active[r] = -1;
+    }
+    if (out.row_lse)
+        for (int i = lane; i < k; i += 32) out.row_lse[r0 + i] = row_lse[r0 + i];
+    // rows the next step has to scan: live slots that have not generated the end token
+    __syncwarp();
+    int n_live = 0, n_done = 0;
+    for (int i0 = 0; i0 < k; i0 += 32) {
+        const int i = i0 + lane;
+        const bool live = i < ns - n_pruned;
+        const bool open = live && a_tok[i] != d.eos_id;
+        n_live += __popc(__ballot_sync(kFullMask, live));
+        n_done += __popc(__ballot_sync(kFullMask, live && !open));
+        const unsigned bal = __ballot_sync(kFullMask, open);
+        int base = 0;
+        if (lane == 0 && bal) base = atomicAdd(open_count, __popc(bal));
+        base = __shfl_sync(kFullMask, base, 0);
+        if (open) open_list[base + __popc(bal & ((1u << lane) - 1u))] = r0 + i;
+    }
+    // Section 4's stopping rule (everything on the beam completed) and Section 6.4's early stopping (something is)
+    if (out.stop && lane == 0)
+        out.stop[b] = (n_live > 0 && n_done == n_live ? DBA_STOP_ALL_COMPLETED : 0) | (n_done > 0 ? DBA_STOP_SOME_COMPLETED : 0);
+}
+
+}  // namespace dba

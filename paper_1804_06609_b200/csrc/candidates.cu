@@ -1,8 +1,10 @@
-// Candidate kernel (Algorithm 2 up to the call of ALLOCATE; Section 3.1; Section 3.3's end-token rule).
+// Candidate kernel (Algorithm 2; Section 3.1; Section 3.3's end-token rule), ending with the allocation of
+// Section 3.2 (allocate_device.cuh) by one of its warps.
 // One CTA per sentence.  Builds the candidate set from (1) the k best cells of the k x V score matrix,
 // (2) every token that advances an open hypothesis through its constraints and (3) every live
 // hypothesis' best token, updates the constraint marks of each candidate (unwinding a broken phrase),
 // removes duplicates, and hands the candidates over grouped by bank and ordered inside each bank.
+#include "allocate_device.cuh"
 #include "dba_device.cuh"
 #include "dba_internal.h"
 
@@ -19,8 +21,8 @@ struct SortEnt {
 };
 
 struct Layout {   // byte offsets into dynamic shared memory
-    int cons, parent, lse, mask, active, kind, eos_ok, s2_x, rt_score, rt_w, rt_n, rt_ptr, s1_h, s1_i, stage, merged,
-        tmp_score, tmp_w, tmp_x, c_score, c_flat, c_mask, c_active, bank_cnt, sort, total;
+    int cons, parent, lse, mask, active, kind, eos_ok, plen, s2_x, rt_score, rt_w, rt_n, rt_ptr, s1_h, s1_i, stage, merged,
+        tmp_score, tmp_w, tmp_x, c_score, c_flat, c_mask, c_active, order, bank_cnt, sort, total;
     int n_sort;
 };
 
@@ -37,6 +39,7 @@ __host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand
     L.active = o;    o += 4 * k;
     L.kind = o;      o += 4 * k;
     L.eos_ok = o;    o += 4 * k;
+    L.plen = o;      o += 4 * k;
     L.s2_x = o;      o += 4 * k * kMaxC;
     L.rt_score = o;  o += 4 * k * k;
     L.rt_w = o;      o += 4 * k * k;
@@ -55,6 +58,7 @@ __host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand
     L.c_score = o;   o += 4 * max_cand;
     L.c_flat = o;    o += 4 * max_cand;
     L.c_active = o;  o += 4 * max_cand;
+    L.order = o;     o += 4 * max_cand;
     L.bank_cnt = o;  o += 4 * (kMaxC + 1);
     o = align_up(o, 16);
     L.n_sort = next_pow2(max_cand);
@@ -81,9 +85,9 @@ __device__ __forceinline__ uint64_t merge_top32(uint64_t a, uint64_t b, int lane
 // 48 registers: two CTAs of 672 threads (a warp per row at k = 20, and one more) fit an SM.
 __global__ void __maxnreg__(48)
 candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const SentCons* __restrict__ cons,
-                  Beam cur, ScanOut part, const float* __restrict__ lse_in, float* __restrict__ row_lse,
-                  Cand* __restrict__ cand_out, int32_t* __restrict__ ncand_out, int32_t* __restrict__ bank_count,
-                  uint32_t* __restrict__ status, int32_t* __restrict__ open_count) {
+                  Beam cur, Beam nxt, ScanOut part, const float* __restrict__ lse_in, float* __restrict__ row_lse,
+                  dba_step_out out, int32_t* __restrict__ hist_bp, int32_t* __restrict__ hist_tok,
+                  uint32_t* __restrict__ status, int32_t* __restrict__ open_list, int32_t* __restrict__ open_count) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int k = d.k, V = d.V, K1 = d.K1, S = d.S;
     const int n_threads = blockDim.x, n_warps = n_threads >> 5;
@@ -95,6 +99,8 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     int* s_active = reinterpret_cast<int*>(smem + L.active);
     int* s_kind = reinterpret_cast<int*>(smem + L.kind);      // 0 empty, 1 open, 2 finished
     int* s_eos_ok = reinterpret_cast<int*>(smem + L.eos_ok);
+    int* s_plen = reinterpret_cast<int*>(smem + L.plen);
+    int* s_order = reinterpret_cast<int*>(smem + L.order);   // candidate ids in (bank, score, flat index) order
     float* s2_x = reinterpret_cast<float*>(smem + L.s2_x);    // logit of the token at constraint position j of row h, if it advances h
     float* rt_score = reinterpret_cast<float*>(smem + L.rt_score);
     int* rt_w = reinterpret_cast<int*>(smem + L.rt_w);
@@ -127,6 +133,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         s_parent[tid] = ps;
         s_mask[tid] = cur.mask[r0 + tid];
         s_active[tid] = cur.active[r0 + tid];
+        s_plen[tid] = cur.len[r0 + tid];
         s_kind[tid] = ps == neg_inf() ? 0 : (tk == d.eos_id ? 2 : 1);
         rt_ptr[tid] = 0;
         rt_n[tid] = 0;
@@ -162,7 +169,6 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     // Up to here only what earlier steps left behind was read (the row scan waited for them before it let
     // this kernel start); from here on the row scan's own results are needed.
     grid_dependency_wait();
-    if (tid == 0 && blockIdx.x == 0) *open_count = 0;   // the allocation kernel rebuilds the list of open rows
     __syncthreads();
     const int C = sc.C;
     if (tid < k) s_eos_ok[tid] = __popcll(s_mask[tid]) >= C;   // Section 3.3: end token only once all are met
@@ -489,8 +495,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
                 const SortEnt o = ent[j];
                 rank += o.hi < me.hi || (o.hi == me.hi && o.lo < me.lo);
             }
-            Cand c; c.score = c_score[tid]; c.flat = c_flat[tid]; c.mask = c_mask[tid]; c.active = c_active[tid]; c.pad_ = 0;
-            cand_out[(int64_t)b * d.max_cand + rank] = c;
+            s_order[rank] = tid;
         }
     } else if (n_sort <= n_threads) {
         // medium list: bitonic network with one entry per thread; partners less than a warp apart are reached by
@@ -514,11 +519,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
                 if (mine_first != want_first) me = o;
             }
         }
-        if (tid < n) {
-            const int id = me.id;
-            Cand c; c.score = c_score[id]; c.flat = c_flat[id]; c.mask = c_mask[id]; c.active = c_active[id]; c.pad_ = 0;
-            cand_out[(int64_t)b * d.max_cand + tid] = c;
-        }
+        if (tid < n) s_order[tid] = (int)me.id;
     } else {
         for (int size = 2; size <= n_sort; size <<= 1) {
             for (int str = size >> 1; str > 0; str >>= 1) {
@@ -532,14 +533,16 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
                 __syncthreads();
             }
         }
-        for (int i = tid; i < n; i += n_threads) {
-            const int id = ent[i].id;
-            Cand c; c.score = c_score[id]; c.flat = c_flat[id]; c.mask = c_mask[id]; c.active = c_active[id]; c.pad_ = 0;
-            cand_out[(int64_t)b * d.max_cand + i] = c;
-        }
+        for (int i = tid; i < n; i += n_threads) s_order[i] = (int)ent[i].id;
     }
-    if (tid <= kMaxC) bank_count[b * (kMaxC + 1) + tid] = bank_cnt[tid];
-    if (tid == 0) ncand_out[b] = n;
+    // ---- ALLOCATE and the new beam (Section 3.2), by one warp ---------------------------------------------
+    __syncthreads();
+    if (warp == 0) {
+        AllocIn in;
+        in.bank_cnt = bank_cnt; in.order = s_order; in.c_score = c_score; in.c_flat = c_flat; in.c_mask = c_mask;
+        in.c_active = c_active; in.par_kind = s_kind; in.par_len = s_plen;
+        allocate_sentence(d, b, C, in, nxt, row_lse, out, hist_bp, hist_tok, open_list, open_count);
+    }
 }
 
 }  // namespace
@@ -572,14 +575,15 @@ cudaError_t configure_candidates(const Dims& d) {
 }
 
 cudaError_t launch_candidates(const void* logits, int64_t stride, const Dims& d, const SentCons* cons,
-                              const Beam& cur, const ScanOut& part, const float* lse_in, float* row_lse,
-                              Cand* cand, int32_t* ncand, int32_t* bank_count, uint32_t* status,
-                              int32_t* open_count, cudaStream_t st, int* launches) {
+                              const Beam& cur, const Beam& next, const ScanOut& part, const float* lse_in,
+                              float* row_lse, const dba_step_out& out, int32_t* hist_bp, int32_t* hist_tok,
+                              uint32_t* status, int32_t* open_list, int32_t* open_count, cudaStream_t st,
+                              int* launches) {
     const int threads = pick_threads(d, g_smem_limit);
     const size_t smem = (size_t)make_layout(d.k, d.K1, d.S, d.max_cand, threads / 32).total;
     ++*launches;
-    return launch_after(candidates_kernel, dim3(d.B), dim3(threads), smem, st, logits, stride, d, cons, cur, part, lse_in,
-                        row_lse, cand, ncand, bank_count, status, open_count);
+    return launch_after(candidates_kernel, dim3(d.B), dim3(threads), smem, st, logits, stride, d, cons, cur, next, part,
+                        lse_in, row_lse, out, hist_bp, hist_tok, status, open_list, open_count);
 }
 
 }  // namespace dba

@@ -21,12 +21,9 @@ struct dba_handle {
     int32_t* hist_tok;
     ScanOut part;
     float* row_lse;
-    Cand* cand;
-    int32_t* ncand;
-    int32_t* bank_count;
     uint32_t* status;
     int32_t* open_list;            // rows the next step scans, and how many
-    int32_t* open_count;
+    int32_t* open_count;           // two counts: step t reads [t & 1], its last kernel fills [(t + 1) & 1]
     int32_t* fin_tokens; int32_t* fin_len; float* fin_score; int32_t* fin_flags;
     void* stage_logits;            // only with DBA_FLAG_HOST_STAGING
     dba_step_out stage_out;
@@ -37,7 +34,7 @@ struct dba_handle {
     uint64_t launches;
     // optional kernel timing
     bool timing;
-    std::vector<cudaEvent_t> ev;   // 4 events per recorded step
+    std::vector<cudaEvent_t> ev;   // 3 events per recorded step
     int ev_steps;
 };
 
@@ -145,9 +142,6 @@ size_t carve(dba_handle* h, void* base, int32_t max_steps) {
     h->part.top_val = cv.take<float>(items * d.K1);
     h->part.top_idx = cv.take<int32_t>(items * d.K1);
     h->row_lse = cv.take<float>(R);
-    h->cand = cv.take<Cand>((size_t)d.B * d.max_cand);
-    h->ncand = cv.take<int32_t>(d.B);
-    h->bank_count = cv.take<int32_t>((size_t)d.B * (kMaxC + 1));
     h->status = cv.take<uint32_t>(64);
     h->open_list = cv.take<int32_t>(R);
     h->open_count = cv.take<int32_t>(64);
@@ -244,31 +238,28 @@ dba_status dba_step(dba_handle* h, const void* logits_dev, int64_t row_stride_el
     h->launches_tmp = 0;
     cudaEvent_t* ev = nullptr;
     if (h->timing && h->ev_steps < kTimingCap) {
-        if ((int)h->ev.size() < 4 * (h->ev_steps + 1)) {
-            for (int i = 0; i < 4; ++i) {
+        if ((int)h->ev.size() < 3 * (h->ev_steps + 1)) {
+            for (int i = 0; i < 3; ++i) {
                 cudaEvent_t x;
                 if (cudaEventCreate(&x) != cudaSuccess) return DBA_ERR_CUDA;
                 h->ev.push_back(x);
             }
         }
-        ev = &h->ev[4 * h->ev_steps];
+        ev = &h->ev[3 * h->ev_steps];
         h->ev_steps += 1;
     }
     cudaError_t e = cudaSuccess;
     if (ev) e = cudaEventRecord(ev[0], h->stream);
     if (e == cudaSuccess)
-        e = launch_row_scan(logits_dev, row_stride_elems, h->d, cur.score, cur.token, h->open_list, h->open_count,
-                            h->part, h->status, h->sm_count, h->stream, &h->launches_tmp);
+        e = launch_row_scan(logits_dev, row_stride_elems, h->d, cur.score, cur.token, h->open_list,
+                            h->open_count + (h->t & 1), h->open_count + ((h->t + 1) & 1), h->part, h->status,
+                            h->sm_count, h->stream, &h->launches_tmp);
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[1], h->stream);
     if (e == cudaSuccess)
-        e = launch_candidates(logits_dev, row_stride_elems, h->d, h->cons, cur, h->part, row_lse_in_dev, h->row_lse,
-                              h->cand, h->ncand, h->bank_count, h->status, h->open_count, h->stream, &h->launches_tmp);
+        e = launch_candidates(logits_dev, row_stride_elems, h->d, h->cons, cur, nxt, h->part, row_lse_in_dev,
+                              h->row_lse, out, h->hist_bp + (size_t)h->t * h->d.R, h->hist_tok + (size_t)h->t * h->d.R,
+                              h->status, h->open_list, h->open_count + ((h->t + 1) & 1), h->stream, &h->launches_tmp);
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[2], h->stream);
-    if (e == cudaSuccess)
-        e = launch_allocate(h->d, h->cons, cur, nxt, h->cand, h->ncand, h->bank_count, h->row_lse, out,
-                            h->hist_bp + (size_t)h->t * h->d.R, h->hist_tok + (size_t)h->t * h->d.R, h->open_list,
-                            h->open_count, h->stream, &h->launches_tmp);
-    if (ev && e == cudaSuccess) e = cudaEventRecord(ev[3], h->stream);
     h->launches += h->launches_tmp;
     if (e != cudaSuccess) return DBA_ERR_CUDA;
     h->cur ^= 1;
@@ -343,9 +334,9 @@ dba_status dba_timing_read(dba_handle* h, double ms_total[3], int64_t* steps) {
     if (cudaStreamSynchronize(h->stream) != cudaSuccess) return DBA_ERR_CUDA;
     ms_total[0] = ms_total[1] = ms_total[2] = 0.0;
     for (int i = 0; i < h->ev_steps; ++i)
-        for (int j = 0; j < 3; ++j) {
+        for (int j = 0; j < 2; ++j) {
             float ms = 0.f;
-            if (cudaEventElapsedTime(&ms, h->ev[4 * i + j], h->ev[4 * i + j + 1]) != cudaSuccess) return DBA_ERR_CUDA;
+            if (cudaEventElapsedTime(&ms, h->ev[3 * i + j], h->ev[3 * i + j + 1]) != cudaSuccess) return DBA_ERR_CUDA;
             ms_total[j] += ms;
         }
     *steps = h->ev_steps;
@@ -413,8 +404,8 @@ dba_status dba_row_scan(const void* logits_dev, int32_t logit_dtype, int32_t R, 
     e = cudaMemsetAsync(status, 0, 256, stream);
     if (e == cudaSuccess) e = configure_row_scan_tma();
     if (e == cudaSuccess)
-        e = launch_row_scan(logits_dev, row_stride_elems, d, nullptr, nullptr, nullptr, nullptr, part, status, sms, stream,
-                            &launches);
+        e = launch_row_scan(logits_dev, row_stride_elems, d, nullptr, nullptr, nullptr, nullptr, nullptr, part, status, sms,
+                            stream, &launches);
     if (e == cudaSuccess) e = launch_row_merge(d, part, n_top, row_lse_dev, top_val_dev, top_idx_dev, stream, &launches);
     return cuda_fail(e);
 }

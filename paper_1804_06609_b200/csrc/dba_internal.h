@@ -41,15 +41,6 @@ struct Beam {
     int32_t* backptr;
 };
 
-// One candidate as handed from the candidate kernel to the allocation kernel.
-struct Cand {
-    float score;
-    int32_t flat;     // h*V + w
-    uint64_t mask;    // constraint marks after generating w
-    int32_t active;
-    int32_t pad_;
-};
-
 struct Dims {
     int32_t B, k, V, R;
     int32_t K1;        // entries kept per row segment by the scan kernel (k + 2, capped by the segment)
@@ -88,25 +79,26 @@ inline cudaError_t launch_after(void (*kernel)(Params...), dim3 grid, dim3 block
 // `open_score` / `open_token` (may be null): rows whose slot is empty (score -inf) or finished
 // (token == eos) are skipped.
 // `open_list` / `open_count` (may be null): the same set of rows as a compact list in device memory.
+// `zero_count` (may be null): a counter the kernel sets to zero (the count of the list the step's last kernel
+// builds for the next step: the two counts alternate).
 cudaError_t launch_row_scan(const void* logits, int64_t stride, const Dims& d, const float* open_score,
                             const int32_t* open_token, const int32_t* open_list, const int32_t* open_count,
-                            const ScanOut& out, uint32_t* status, int sm_count, cudaStream_t st, int* launches);
+                            int32_t* zero_count, const ScanOut& out, uint32_t* status, int sm_count,
+                            cudaStream_t st, int* launches);
 // streaming (TMA) version: usable when rows start on 16-byte boundaries and segments are whole chunks
 bool row_scan_tma_usable(const void* logits, int64_t stride, const Dims& d);
 cudaError_t configure_row_scan_tma();
 cudaError_t launch_row_scan_tma(const void* logits, int64_t stride, const Dims& d, const int32_t* open_list,
-                                const int32_t* open_count, const ScanOut& out, uint32_t* status, int sm_count,
-                                cudaStream_t st);
+                                const int32_t* open_count, int32_t* zero_count, const ScanOut& out, uint32_t* status,
+                                int sm_count, cudaStream_t st);
 cudaError_t launch_row_merge(const Dims& d, const ScanOut& part, int n_top, float* row_lse, float* top_val,
                              int32_t* top_idx, cudaStream_t st, int* launches);
+// candidates, allocation and the new beam (one kernel); appends the new beam's open rows to open_list / open_count
 cudaError_t launch_candidates(const void* logits, int64_t stride, const Dims& d, const SentCons* cons,
-                              const Beam& cur, const ScanOut& part, const float* lse_in, float* row_lse,
-                              Cand* cand, int32_t* ncand, int32_t* bank_count, uint32_t* status,
-                              int32_t* open_count, cudaStream_t st, int* launches);
-cudaError_t launch_allocate(const Dims& d, const SentCons* cons, const Beam& cur, const Beam& next,
-                            const Cand* cand, const int32_t* ncand, const int32_t* bank_count,
-                            const float* row_lse, const dba_step_out& out, int32_t* hist_bp, int32_t* hist_tok,
-                            int32_t* open_list, int32_t* open_count, cudaStream_t st, int* launches);
+                              const Beam& cur, const Beam& next, const ScanOut& part, const float* lse_in,
+                              float* row_lse, const dba_step_out& out, int32_t* hist_bp, int32_t* hist_tok,
+                              uint32_t* status, int32_t* open_list, int32_t* open_count, cudaStream_t st,
+                              int* launches);
 cudaError_t launch_reset(const Dims& d, const Beam& beam, int32_t* open_list, int32_t* open_count,
                          cudaStream_t st, int* launches);
 cudaError_t launch_finalize(const Dims& d, const Beam& beam, const int32_t* hist_bp, const int32_t* hist_tok,

@@ -43,11 +43,12 @@ template <typename T>
 __global__ void __launch_bounds__(kScanThreads)
 row_scan_generic_kernel(const T* __restrict__ logits, int64_t stride, int V, int S, int seg_len, int K1,
                         int eos, const float* __restrict__ open_score, const int32_t* __restrict__ open_token,
-                        float* __restrict__ part_m, float* __restrict__ part_s,
+                        int32_t* __restrict__ zero_count, float* __restrict__ part_m, float* __restrict__ part_s,
                         float* __restrict__ top_val, int32_t* __restrict__ top_idx) {
     __shared__ float smf[kScanThreads / 32];
     __shared__ uint64_t smu[kScanThreads / 32];
     const int item = blockIdx.x;
+    if (zero_count && item == 0 && threadIdx.x == 0) *zero_count = 0;
     const int r = item / S, g = item - r * S;
     if (open_score) {
         if (open_score[r] == neg_inf() || open_token[r] == eos) return;   // empty or finished slot
@@ -138,19 +139,20 @@ void plan_segments(Dims& d, int sm_count) {
 
 cudaError_t launch_row_scan(const void* logits, int64_t stride, const Dims& d, const float* open_score,
                             const int32_t* open_token, const int32_t* open_list, const int32_t* open_count,
-                            const ScanOut& out, uint32_t* status, int sm_count, cudaStream_t st, int* launches) {
+                            int32_t* zero_count, const ScanOut& out, uint32_t* status, int sm_count, cudaStream_t st,
+                            int* launches) {
     ++*launches;
     if (row_scan_tma_usable(logits, stride, d))
-        return launch_row_scan_tma(logits, stride, d, open_list, open_count, out, status, sm_count, st);
+        return launch_row_scan_tma(logits, stride, d, open_list, open_count, zero_count, out, status, sm_count, st);
     const int items = d.R * d.S;
     if (d.dtype == DBA_F32)
         row_scan_generic_kernel<float><<<items, kScanThreads, 0, st>>>(
-            (const float*)logits, stride, d.V, d.S, d.seg_len, d.K1, d.eos_id, open_score, open_token, out.m,
-            out.s, out.top_val, out.top_idx);
+            (const float*)logits, stride, d.V, d.S, d.seg_len, d.K1, d.eos_id, open_score, open_token, zero_count,
+            out.m, out.s, out.top_val, out.top_idx);
     else
         row_scan_generic_kernel<__nv_bfloat16><<<items, kScanThreads, 0, st>>>(
             (const __nv_bfloat16*)logits, stride, d.V, d.S, d.seg_len, d.K1, d.eos_id, open_score, open_token,
-            out.m, out.s, out.top_val, out.top_idx);
+            zero_count, out.m, out.s, out.top_val, out.top_idx);
     return cudaGetLastError();
 }
 

@@ -81,6 +81,7 @@ struct Params {
     int R;
     const int32_t* open_list;   // rows to scan (null: all R rows)
     const int32_t* open_count;  // number of entries of open_list (device memory)
+    int32_t* zero_count;        // set to zero here: the count of the list the step's last kernel builds (may be null)
     float* part_m; float* part_s; float* top_val; int32_t* top_idx;
     uint32_t* status;
 };
@@ -309,7 +310,10 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
     }
     __syncthreads();
     grid_dependency_wait();      // the list of open rows comes from the previous step's last kernel
-    if (tid == 0) allow_dependents();
+    if (tid == 0) {
+        if (blockIdx.x == 0 && p.zero_count) *p.zero_count = 0;     // before the next kernel can start
+        allow_dependents();
+    }
 
     if (warp == kWarpProd) {
         // ------------------------------------------------------------------ producer
@@ -654,11 +658,11 @@ cudaError_t configure_row_scan_tma() {
 }
 
 cudaError_t launch_row_scan_tma(const void* logits, int64_t stride, const Dims& d, const int32_t* open_list,
-                                const int32_t* open_count, const ScanOut& out, uint32_t* status, int sm_count,
-                                cudaStream_t st) {
+                                const int32_t* open_count, int32_t* zero_count, const ScanOut& out, uint32_t* status,
+                                int sm_count, cudaStream_t st) {
     Params p;
     p.logits = logits; p.stride = stride; p.V = d.V; p.S = d.S; p.seg_len = d.seg_len; p.K1 = d.K1; p.R = d.R;
-    p.open_list = open_list; p.open_count = open_count;
+    p.open_list = open_list; p.open_count = open_count; p.zero_count = zero_count;
     p.part_m = out.m; p.part_s = out.s; p.top_val = out.top_val; p.top_idx = out.top_idx; p.status = status;
     const int64_t items = (int64_t)d.R * d.S;
     const int grid = (int)(items < sm_count ? items : sm_count);
