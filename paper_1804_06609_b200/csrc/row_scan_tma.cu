@@ -393,11 +393,16 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
                 // the chunk is read from the buffer a second time: held in registers since the maxima, it would
                 // leave the exponentials too few registers to overlap one another
                 const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[slot]) + chunk * kChunkVecs + lane;
+                if (nvec >= kChunkVecs) {
 #pragma unroll
-                for (int i = 0; i < kVecsPerLane; ++i) {
-                    const uint32_t w = Vec<T>::kNegInfWord;
-                    const uint4 vv = i * 32 + lane < nvec ? vec[i * 32] : make_uint4(w, w, w, w);
-                    Vec<T>::exp_sum(vv, L2, C2, a0, a1);
+                    for (int i = 0; i < kVecsPerLane; ++i) Vec<T>::exp_sum(vec[i * 32], L2, C2, a0, a1);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < kVecsPerLane; ++i) {
+                        const uint32_t w = Vec<T>::kNegInfWord;
+                        const uint4 vv = i * 32 + lane < nvec ? vec[i * 32] : make_uint4(w, w, w, w);
+                        Vec<T>::exp_sum(vv, L2, C2, a0, a1);
+                    }
                 }
                 float s0, s1, s2, s3;
                 unpack2(a0, s0, s1); unpack2(a1, s2, s3);
