@@ -153,6 +153,26 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------------------------- replicas
+def replica_workload(wl, rank):
+    """Rank `rank`'s replica of the workload: the same shapes and constraints recipe, its own sentence ids (and
+    hence its own logit streams).  Sentences never interact, so ranks exchange nothing on the data path."""
+    import numpy as np
+    wl.sent_ids = wl.sent_ids + np.int64(rank * wl.B)
+    return wl
+
+
+def job_rate(units_per_rank, seconds_local, world, device):
+    """Whole-job rate: the units all ranks processed over the slowest rank's time (max over ranks)."""
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        t = torch.tensor([seconds_local], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        seconds_local = float(t)
+    return world * units_per_rank / seconds_local, seconds_local
+
+
 # ---------------------------------------------------------------------------------------------- ours
 def run_ours(args):
     import torch
@@ -171,8 +191,7 @@ def run_ours(args):
 
     wl = workload_of(args)
     if world > 1:                                   # replicas: every rank gets its own sentences
-        import numpy as np
-        wl.sent_ids = wl.sent_ids + np.int64(rank * wl.B)
+        wl = replica_workload(wl, rank)
     esize = 2 if wl.dtype == "bf16" else 4
     step_bytes = wl.R * wl.V * esize
     free, _ = torch.cuda.mem_get_info(dev)
@@ -221,9 +240,8 @@ def run_ours(args):
     sampler.stop_flag = True; sampler.join()
     ms = e0.elapsed_time(e1)
     launches = st.launch_count() - launches0
-    if world > 1:
-        tms = torch.tensor([ms], device=dev); dist.all_reduce(tms, op=dist.ReduceOp.MAX); ms = float(tms)
-    value = world * args.steps / (ms / 1e3)
+    value, secs = job_rate(args.steps, ms / 1e3, world, dev)
+    ms = secs * 1e3
 
     # --- per-kernel time of the same replay (events inside the library, on its stream) -----------------
     st.timing_enable(True)
@@ -265,9 +283,7 @@ def run_ours(args):
     replay_host(args.e2e_steps)
     torch.cuda.synchronize(dev)
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        te = torch.tensor([e2e_s], device=dev); dist.all_reduce(te, op=dist.ReduceOp.MAX); e2e_s = float(te)
-    e2e_value = world * args.e2e_steps / e2e_s
+    e2e_value, e2e_s = job_rate(args.e2e_steps, e2e_s, world, dev)
 
     if rank != 0:
         if world > 1:
