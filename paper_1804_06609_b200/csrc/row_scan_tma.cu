@@ -318,17 +318,29 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
     if (warp == kWarpProd) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            ItemIter it(p, (int)sizeof(T));
+            ItemIter it(p, (int)sizeof(T)), ahead = it;
             bool ok = true;
+            // the row numbers come from a list in global memory: they are asked for kSlots items ahead, so that
+            // no copy waits for one (the first kSlots loads overlap one another)
+            int rows[kSlots];
+#pragma unroll
+            for (int j = 0; j < kSlots; ++j) { rows[j] = ahead.valid() ? ahead.row(p.open_list) : 0; ahead.next(); }
 #pragma unroll 1
-            for (; it.valid(); it.next()) {
-                const uint32_t slot = it.slot();
-                const int row = it.row(p.open_list);
-                if (!mbar_try_wait(smem_u32(&sm.loaded[slot]), it.slot_phase() ^ 1u) &&
-                    !mbar_wait(smem_u32(&sm.loaded[slot]), it.slot_phase() ^ 1u, abort_flag)) { ok = false; break; }
-                const char* src = (const char*)p.logits + ((int64_t)row * p.stride + (int64_t)it.seg() * p.seg_len) * (int64_t)sizeof(T);
-                mbar_expect_tx(smem_u32(&sm.full[slot]), (uint32_t)it.bytes());
-                bulk_load(smem_u32(sm.ring[slot]), src, (uint32_t)it.bytes(), smem_u32(&sm.full[slot]));
+            while (ok && it.valid()) {
+#pragma unroll
+                for (int j = 0; j < kSlots; ++j) {          // item n uses slot n % kSlots = j
+                    if (!it.valid()) break;
+                    const uint32_t slot = j;
+                    const int row = rows[j];
+                    rows[j] = ahead.valid() ? ahead.row(p.open_list) : 0;
+                    ahead.next();
+                    if (!mbar_try_wait(smem_u32(&sm.loaded[slot]), it.slot_phase() ^ 1u) &&
+                        !mbar_wait(smem_u32(&sm.loaded[slot]), it.slot_phase() ^ 1u, abort_flag)) { ok = false; break; }
+                    const char* src = (const char*)p.logits + ((int64_t)row * p.stride + (int64_t)it.seg() * p.seg_len) * (int64_t)sizeof(T);
+                    mbar_expect_tx(smem_u32(&sm.full[slot]), (uint32_t)it.bytes());
+                    bulk_load(smem_u32(sm.ring[slot]), src, (uint32_t)it.bytes(), smem_u32(&sm.full[slot]));
+                    it.next();
+                }
             }
             if (!ok) {   // winding down: let the copies already issued land before the CTA leaves
                 const uint32_t n = it.n_item;
