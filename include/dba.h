@@ -174,6 +174,15 @@ dba_status dba_finalize(dba_handle* h, int32_t* tokens_host, int32_t* len_host, 
 dba_status dba_timing_enable(dba_handle* h, int32_t on);
 dba_status dba_timing_read(dba_handle* h, double ms_total[3], int64_t* steps);
 
+/*
+ * Diagnostic counters of the handle's device status block (never an error).  Synchronises the stream.
+ *   counters[0]  row segments whose K1 best entries the row scan had to find by a second, slow pass over global
+ *                memory, because more entries tied at its selection bound than its lists hold (long runs of
+ *                equal logits).  Results are exact either way; a large count explains a slow step.
+ *   counters[1..3]  reserved, 0.
+ */
+dba_status dba_counters(dba_handle* h, uint32_t counters[4]);
+
 /* Number of kernels this handle has launched so far (for accounting in benchmarks). */
 uint64_t dba_launch_count(const dba_handle* h);
 

@@ -15,7 +15,7 @@ F32, BF16 = 0, 1
 FLAG_ADJUST_OFF, FLAG_LENGTH_NORM, FLAG_HOST_STAGING = 1, 2, 4
 
 EXPORTS = ["dba_workspace_bytes", "dba_init", "dba_reset", "dba_step", "dba_step_host", "dba_finalize",
-           "dba_timing_enable", "dba_timing_read", "dba_launch_count", "dba_destroy", "dba_status_string", "dba_row_scan_scratch_bytes", "dba_row_scan",
+           "dba_timing_enable", "dba_timing_read", "dba_counters", "dba_launch_count", "dba_destroy", "dba_status_string", "dba_row_scan_scratch_bytes", "dba_row_scan",
            "dba_row_scan_static", "dba_row_scan_static_max_bytes"]
 
 
@@ -56,6 +56,7 @@ def lib():
         L.dba_finalize.argtypes = [vp, vp, vp, vp, vp]
         L.dba_timing_enable.argtypes = [vp, C.c_int32]
         L.dba_timing_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+        L.dba_counters.argtypes = [vp, C.POINTER(C.c_uint32)]
         L.dba_launch_count.argtypes = [vp]
         L.dba_launch_count.restype = C.c_uint64
         L.dba_destroy.argtypes = [vp]
@@ -174,6 +175,12 @@ class DbaStepper:
         ms = (C.c_double * 3)(); n = C.c_int64()
         _check(lib().dba_timing_read(self._h, ms, C.byref(n)), "dba_timing_read")
         return list(ms), n.value
+
+    def counters(self):
+        """Diagnostic counters: [row segments ranked by the slow second pass, 0, 0, 0]."""
+        out = (C.c_uint32 * 4)()
+        _check(lib().dba_counters(self._h, out), "dba_counters")
+        return list(out)
 
     def launch_count(self):
         return int(lib().dba_launch_count(self._h))

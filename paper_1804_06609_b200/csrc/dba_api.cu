@@ -344,6 +344,16 @@ dba_status dba_timing_read(dba_handle* h, double ms_total[3], int64_t* steps) {
     return DBA_OK;
 }
 
+dba_status dba_counters(dba_handle* h, uint32_t counters[4]) {
+    if (!h || !counters) return DBA_ERR_INVALID_ARG;
+    uint32_t words[4] = {};
+    cudaError_t e = cudaMemcpyAsync(words, h->status, sizeof words, cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) return DBA_ERR_CUDA;
+    counters[0] = words[kStatusWordRescans]; counters[1] = counters[2] = counters[3] = 0;
+    return DBA_OK;
+}
+
 uint64_t dba_launch_count(const dba_handle* h) { return h ? h->launches : 0; }
 
 void dba_destroy(dba_handle* h) {

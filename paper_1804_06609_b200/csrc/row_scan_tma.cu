@@ -256,7 +256,8 @@ struct ItemIter {
     __device__ int chunk_vecs(int c) const { return min(kChunkBytes, bytes_ - c * kChunkBytes) >> 4; }
     // Warps whose 32 lanes all hold data report (they are the first report_warps() of the team).  Each reports
     // the maxima of G = 32 >> tap groups of lanes, where tap is the number of butterfly steps taken before the
-    // values are recorded; G is the smallest of 4, 8, 16, 32 that gives at least K1 reports.
+    // values are recorded; G is the largest of 4, 8, 16, 32 that keeps the item at 64 reports or fewer, or, if
+    // that is fewer than K1, the smallest that gives K1.
     // tap < 0: no usable bound, every entry is kept.
     __device__ int report_warps() const {
         const int nvec = bytes_ >> 4;
@@ -265,7 +266,10 @@ struct ItemIter {
     __device__ int report_tap(int K1) const {
         const int warps = report_warps();
         if (warps == 0) return -1;
-        for (int tap = 3; tap >= 0; --tap)             // G = 4, 8, 16, 32
+        // as many reports as the selector's fast path takes (64): the more reports, the tighter the bound
+        for (int tap = 0; tap <= 3; ++tap)             // G = 32, 16, 8, 4
+            if ((32 >> tap) * warps <= 64) { if ((32 >> tap) * warps >= K1) return tap; break; }
+        for (int tap = 3; tap >= 0; --tap)             // more than 64 reports are needed: G = 4, 8, 16, 32
             if ((32 >> tap) * warps >= K1) return (32 >> tap) * warps <= kRepCap ? tap : -1;
         return -1;
     }

@@ -244,6 +244,37 @@ def test_scores_that_round_together_across_the_row_cut(dba):
     assert len(np.unique(sc)) < k                                   # the case really had equal scores
 
 
+@pytest.mark.parametrize("B", [8, 30])
+def test_the_row_scan_needs_no_second_pass_on_benchmark_shaped_rows(dba, B):
+    """A performance guard: the scan's selection bound must be tight enough on Zipf-shaped bf16 rows that no
+    row segment is ranked again from global memory (that pass costs about as much as scanning 150 rows), also
+    for the short segments a small batch gets (few warps per segment, hence few reports)."""
+    from synth_inputs.gpu import GpuLogitStream
+    wl = make_workload("serving", B=B, steps=12)
+    st = _stepper(dba, wl)
+    gen = GpuLogitStream(wl)
+    tok = torch.zeros(wl.R, dtype=torch.int32, device="cuda"); tok[::wl.k] = 1
+    mask = torch.zeros(wl.R, dtype=torch.int64, device="cuda")
+    for t in range(wl.steps):
+        out = st.step(gen.step_logits(t, tok, mask))
+        tok, mask = out["token"].clone(), out["met_mask"].clone()
+    assert st.counters()[0] == 0
+    st.close()
+
+
+def test_long_runs_of_equal_logits_take_the_second_pass_and_stay_exact(dba):
+    wl = _custom("flat", B=2, k=20, V=64000, steps=2, dtype="bf16", constraints=[[[5, 6]], [[7]]])
+    st = _stepper(dba, wl)
+    orc = O.Batch(wl.k, wl.V, wl.steps, wl.constraints)
+    for t in range(wl.steps):
+        x = np.full((wl.R, wl.V), 0x3F80, np.uint16)          # every logit 1.0: everything ties at the bound
+        lse_o = orc.step(x)
+        out = st.step(to_device_logits(x, wl), row_lse_in=torch.from_numpy(lse_o).cuda())
+        assert_beam_equal(gpu_beam(out), orc.beam(), f"flat step {t}")
+    assert st.counters()[0] > 0
+    st.close()
+
+
 def test_step_host_equals_step_and_reset_replays(dba):
     wl = make_workload("ragged", B=4, V=2000, steps=12)
     gen = LogitStream(wl)
