@@ -116,7 +116,7 @@ void fill_dims(const dba_config* c, const Shape& sh, Dims* d) {
     d->dtype = c->logit_dtype; d->flags = c->flags;
     d->prune = c->prune_threshold > 0.f ? c->prune_threshold : 0.f;
     d->max_cand = c->k * (sh.max_phrases + 2);
-    d->K1 = c->k + 2; d->S = kMaxSeg; d->seg_len = 0;   // S is an upper bound until plan_segments runs
+    d->K1 = c->k + 2; d->S = max_segments(c->V, c->logit_dtype); d->seg_len = 0;   // an upper bound until plan_segments runs
 }
 
 Beam carve_beam(Carver& cv, int R) {
@@ -127,11 +127,11 @@ Beam carve_beam(Carver& cv, int R) {
     return b;
 }
 
-// Lays the handle's arrays out in the workspace; sizes use the upper bound kMaxSeg for the segment count.
+// Lays the handle's arrays out in the workspace; sizes use the upper bound max_segments for the segment count.
 size_t carve(dba_handle* h, void* base, int32_t max_steps) {
     Carver cv(base);
     const Dims& d = h->d;
-    const size_t R = d.R, items = (size_t)d.R * kMaxSeg;
+    const size_t R = d.R, items = (size_t)d.R * max_segments(d.V, d.dtype);
     h->cons = cv.take<SentCons>(d.B);
     h->beam[0] = carve_beam(cv, d.R);
     h->beam[1] = carve_beam(cv, d.R);
@@ -380,7 +380,7 @@ dba_status dba_row_scan_scratch_bytes(int32_t R, int32_t V, int32_t n_top, int32
     if (logit_dtype != DBA_F32 && logit_dtype != DBA_BF16) return DBA_ERR_INVALID_ARG;
     if (n_top > kMaxTop) return DBA_ERR_UNSUPPORTED;
     Carver cv(nullptr);
-    const size_t items = (size_t)R * kMaxSeg;
+    const size_t items = (size_t)R * max_segments(V, logit_dtype);
     cv.take<float>(items); cv.take<float>(items); cv.take<float>(items * n_top); cv.take<int32_t>(items * n_top);
     cv.take<uint32_t>(64);
     *bytes = (cv.off + 255) / 256 * 256;
@@ -404,7 +404,7 @@ dba_status dba_row_scan(const void* logits_dev, int32_t logit_dtype, int32_t R, 
     plan_segments(d, sms);
     d.K1 = n_top;
     Carver cv(scratch_dev);
-    const size_t items = (size_t)R * kMaxSeg;
+    const size_t items = (size_t)R * max_segments(V, logit_dtype);
     ScanOut part;
     part.m = cv.take<float>(items); part.s = cv.take<float>(items);
     part.top_val = cv.take<float>(items * n_top); part.top_idx = cv.take<int32_t>(items * n_top);

@@ -10,7 +10,8 @@ namespace dba {
 constexpr int kMaxK = 64;          // beam size limit
 constexpr int kMaxC = 64;          // constraint tokens per sentence (one bit each in a 64-bit mask)
 constexpr int kMaxTop = kMaxK + 2; // entries kept per row: k, one for a masked end token, one sentinel
-constexpr int kMaxSeg = 8;         // row segments scanned by different CTAs
+constexpr int kMaxSeg = 8;         // row segments scanned by different CTAs: as far as short rows are split up
+constexpr int kMaxSegLong = 24;    // segments of a row too long for kMaxSeg full-length segments (up to 1 MiB)
 
 // device status word bits (sticky; read by dba_finalize)
 constexpr uint32_t kStatusTimeout = 1u;    // a bounded wait on an mbarrier gave up
@@ -111,5 +112,7 @@ cudaError_t configure_candidates(const Dims& d);
 
 // Chooses S and seg_len for a row of V elements when R rows are scanned (fills d.S, d.seg_len, d.K1).
 void plan_segments(Dims& d, int sm_count);
+// The most segments plan_segments can choose for such rows: what the per-segment arrays are sized for.
+int max_segments(int V, int dtype);
 
 }  // namespace dba

@@ -118,23 +118,32 @@ __global__ void row_merge_kernel(int R, int S, int K1, int n_top, const float* _
 }  // namespace
 
 void plan_segments(Dims& d, int sm_count) {
-    // Segments are whole 4 KB chunks, at most twelve of them (what one team of the streaming kernel holds);
+    // Segments are whole 4 KB chunks, at most eleven of them (what one team of the streaming kernel holds);
     // shorter segments when there are few rows, so that every SM has several (row, segment) items to work on,
     // but never more than kMaxSeg segments per row.
     const int es = d.dtype == DBA_F32 ? 4 : 2;
     const int chunk_elems = 4096 / es;
     const int row_chunks = (d.V + chunk_elems - 1) / chunk_elems;
     auto segs = [&](int c) { return (row_chunks + c - 1) / c; };
-    int chunks = 12;
-    while (segs(chunks) > kMaxSeg) chunks *= 2;                       // very long rows: longer segments
-    if (chunks == 12) {
-        chunks = (row_chunks + segs(12) - 1) / segs(12);             // same number of segments, evened out
+    int chunks;
+    if (segs(11) > kMaxSeg) {                                         // long rows: full-length segments, more of them;
+        chunks = 11;                                                  // beyond kMaxSegLong: longer ones (generic kernel)
+        while (segs(chunks) > kMaxSegLong) chunks *= 2;
+    } else {
+        chunks = (row_chunks + segs(11) - 1) / segs(11);             // as few segments as possible, evened out
         while (chunks > 1 && (int64_t)d.R * segs(chunks) < 4LL * sm_count && segs((chunks + 1) / 2) <= kMaxSeg)
             chunks = (chunks + 1) / 2;
     }
     d.seg_len = chunks * chunk_elems;
     d.S = segs(chunks);
     d.K1 = d.k + 2;
+}
+
+int max_segments(int V, int dtype) {
+    const int chunk_elems = 4096 / (dtype == DBA_F32 ? 4 : 2);
+    const int row_chunks = (V + chunk_elems - 1) / chunk_elems;
+    const int full = (row_chunks + 10) / 11;
+    return full <= kMaxSeg ? kMaxSeg : (full <= kMaxSegLong ? full : kMaxSegLong);
 }
 
 cudaError_t launch_row_scan(const void* logits, int64_t stride, const Dims& d, const float* open_score,

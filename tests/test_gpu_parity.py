@@ -71,7 +71,8 @@ def _rows(kind, R, V, rng):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("kind", ["normal", "ascending", "descending", "constant", "quantised", "holes", "signed_zero"])
-@pytest.mark.parametrize("V,n_top", [(1, 3), (7, 7), (1000, 7), (4099, 22), (32000, 12), (64000, 22), (20011, 66)])
+@pytest.mark.parametrize("V,n_top", [(1, 3), (7, 7), (1000, 7), (4099, 22), (32000, 12), (64000, 22), (20011, 66),
+                                      (24576, 12), (150000, 22), (262144, 7)])
 def test_row_scan_matches_oracle(dba, dtype, kind, V, n_top):
     from synth_inputs.logits import to_bf16_bits
     rng = np.random.default_rng(V + n_top)
@@ -242,6 +243,16 @@ def test_scores_that_round_together_across_the_row_cut(dba):
         assert_beam_equal(gpu_beam(out), orc.beam(), f"collapse step {t}")
     sc = orc.beam()["score"]
     assert len(np.unique(sc)) < k                                   # the case really had equal scores
+
+
+def test_step_parity_on_rows_of_more_than_eight_segments(dba):
+    """Rows longer than eight full segments (Transformer-sized vocabularies in fp32): up to 24 segments per row."""
+    wl = _custom("long_rows", B=2, k=4, V=150000, steps=5, constraints=[[[5, 6], [70000]], [[149999]]])
+    st = _stepper(dba, wl)
+    orc, worst = lockstep(wl, st, threads=2)
+    assert_finalize_equal(st, orc)
+    assert st.counters()[0] == 0
+    st.close()
 
 
 @pytest.mark.parametrize("B", [8, 30])
