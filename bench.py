@@ -35,6 +35,9 @@ def parse():
     ap.add_argument("--workload", default="serving")
     ap.add_argument("--C", type=int, default=None, help="constraint count of the 'scaling' workload")
     ap.add_argument("--B", type=int, default=None, help="fewer sentences than the workload has (for profiling a small case)")
+    ap.add_argument("--gbs-base", type=int, default=None,
+                    help="grid-beam-search simulation of the paper's Section 5 on the 'scaling' workload: beam "
+                         "b*(C+1) for this base beam b, bank adjustment off")
     ap.add_argument("--stream-steps", type=int, default=None, help="keep only the first steps of the stream resident")
     ap.add_argument("--e2e-steps", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -101,6 +104,8 @@ class ClockSampler(threading.Thread):
 def workload_of(args):
     from synth_inputs import make_workload
     kw = {"B": args.B} if args.B else {}
+    if args.gbs_base:                       # Section 5: every bank has its own b slots, so the beam grows with C
+        kw["k"] = args.gbs_base * ((args.C if args.C is not None else 10) + 1)
     return make_workload(args.workload, C=args.C, **kw)
 
 
@@ -198,8 +203,9 @@ def run_ours(args):
     T = int(max(1, min(wl.steps, (free * 0.6) // step_bytes, args.stream_steps or wl.steps)))
     # rotate enough distinct step buffers that consecutive steps never find their input in L2
     gen = GpuLogitStream(wl, dev)
+    cfg_flags = pkg.FLAG_ADJUST_OFF if args.gbs_base else 0
     st = pkg.DbaStepper(wl.B, wl.k, wl.V, wl.steps, constraints=wl.constraints,
-                        dtype=pkg.BF16 if wl.dtype == "bf16" else pkg.F32, device=dev)
+                        dtype=pkg.BF16 if wl.dtype == "bf16" else pkg.F32, device=dev, flags=cfg_flags)
     logits = torch.empty(T, wl.R, wl.V, dtype=gen.tdtype, device=dev)
 
     # --- untimed: generate the stream in closed loop, count the rows that are open at each step -------
@@ -265,7 +271,7 @@ def run_ours(args):
     Th = min(T, 8)
     ste = pkg.DbaStepper(wl.B, wl.k, wl.V, wl.steps, constraints=wl.constraints,
                          dtype=pkg.BF16 if wl.dtype == "bf16" else pkg.F32, device=dev,
-                         flags=pkg.FLAG_HOST_STAGING)
+                         flags=pkg.FLAG_HOST_STAGING | cfg_flags)
     host = torch.empty(Th, wl.R, wl.V, dtype=gen.tdtype, pin_memory=True)
     host.copy_(logits[:Th])
     host_out = ste.new_outputs(host=True)
@@ -307,7 +313,8 @@ def run_ours(args):
                    "completed_sentences": completed,
                    "l2": f"inputs larger than L2: {step_bytes >> 20} MiB of logits per step, {T} step buffers"
                          if step_bytes > L2_BYTES else f"{T} rotating step buffers, {T * step_bytes >> 20} MiB in all",
-                   "parallelism": "replicas" if world > 1 else "single GPU"},
+                   "parallelism": "replicas" if world > 1 else "single GPU",
+                   **({"gbs_simulation": {"base_beam": args.gbs_base, "beam": wl.k, "bank_adjustment": "off"}} if args.gbs_base else {})},
         "hyp_steps_per_sec": value * wl.R,
         "kernel_ms": {"row_scan": scan_ms, "candidates_and_allocation": kt[1] / ksteps},
         "roofline": {"bound": "hbm", "kernel": "row_scan", "achieved": achieved, "peak": peak, "unit": "GB/s",

@@ -46,8 +46,8 @@ constexpr int kWarpRank = kNR;                 // first ranking warp
 constexpr int kWarpProd = 2 * kNR;             // the producer's warp
 constexpr int kWarpCons = 2 * kNR + 1;         // first consumer warp
 constexpr int kThreads = 32 * (kWarpCons + kNC);
-constexpr int kHitCap = 96;                    // cells reaching the bound that one item may have
-constexpr int kKeyCap = 128;                   // entries at or above the bound that one item may hold
+constexpr int kHitCap = 192;                   // cells reaching the bound that one item may have (three per wanted entry at K1 = 66)
+constexpr int kKeyCap = 256;                   // entries at or above the bound that one item may hold
 constexpr int kRepCap = 192;                   // reports of one item (11 warps x 16 groups fit)
 constexpr long long kWaitClocks = 2000000000LL;            // about a second: a wait this long has failed
 constexpr float kLog2e = 1.44269502162933349609375f;        // fl32(log2(e))

@@ -255,13 +255,14 @@ def test_step_parity_on_rows_of_more_than_eight_segments(dba):
     st.close()
 
 
-@pytest.mark.parametrize("B", [8, 30])
-def test_the_row_scan_needs_no_second_pass_on_benchmark_shaped_rows(dba, B):
+@pytest.mark.parametrize("B,k", [(8, 20), (30, 20), (6, 60)])
+def test_the_row_scan_needs_no_second_pass_on_benchmark_shaped_rows(dba, B, k):
     """A performance guard: the scan's selection bound must be tight enough on Zipf-shaped bf16 rows that no
     row segment is ranked again from global memory (that pass costs about as much as scanning 150 rows), also
-    for the short segments a small batch gets (few warps per segment, hence few reports)."""
+    for the short segments a small batch gets (few warps per segment, hence few reports) and for a wide beam
+    (three times as many entries wanted per segment)."""
     from synth_inputs.gpu import GpuLogitStream
-    wl = make_workload("serving", B=B, steps=12)
+    wl = make_workload("serving", B=B, k=k, steps=12)
     st = _stepper(dba, wl)
     gen = GpuLogitStream(wl)
     tok = torch.zeros(wl.R, dtype=torch.int32, device="cuda"); tok[::wl.k] = 1
