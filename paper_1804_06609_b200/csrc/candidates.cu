@@ -195,10 +195,24 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         const float mg = lane < S ? part.m[r * S + lane] : neg_inf();
         const float sg = lane < S ? part.s[r * S + lane] : 0.f;
         const float lse_given = lse_in ? lse_in[r] : 0.f;
-        for (int e = lane; e < n_ent; e += 32) {
-            const int ix = part.top_idx[(int64_t)r * n_ent + e];
-            const float xv = part.top_val[(int64_t)r * n_ent + e];
-            (S == 1 ? merged : stage)[e] = ix >= 0 ? row_key(xv, ix) : 0ull;
+        {   // four loads of each array in flight before the first key is stored (the stores would hold them back)
+            uint64_t* dst = S == 1 ? merged : stage;
+            const int32_t* gi = part.top_idx + (int64_t)r * n_ent;
+            const float* gv = part.top_val + (int64_t)r * n_ent;
+            for (int e0 = lane; e0 < n_ent; e0 += 128) {
+                int ix[4]; float xv[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int e = e0 + 32 * q;
+                    ix[q] = e < n_ent ? __ldg(gi + e) : -1;
+                    xv[q] = e < n_ent ? __ldg(gv + e) : 0.f;
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int e = e0 + 32 * q;
+                    if (e < n_ent) dst[e] = ix[q] >= 0 ? row_key(xv[q], ix[q]) : 0ull;
+                }
+            }
         }
         // row normaliser from the segment partials: lane g holds segment g (S <= 8), fixed reduction order
         float lse;
