@@ -8,7 +8,7 @@ namespace dba {
 
 constexpr unsigned kFullMask = 0xffffffffu;
 
-// Programmatic dependent launch: the three kernels of a step follow one another on a stream.  A kernel
+// Programmatic dependent launch: the kernels of successive steps follow one another on a stream.  A kernel
 // launched with launch_after() may start while its predecessor is still running; it must not touch what the
 // predecessor produces (or still reads and this kernel writes) before grid_dependency_wait() returns, which
 // is when the predecessor has finished and its writes are visible.  allow_dependents() lets the successor's
