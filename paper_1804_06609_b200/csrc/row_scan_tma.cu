@@ -284,7 +284,7 @@ __device__ __noinline__ void rank_from_global(const T* src, int e0, int e1, int 
 #pragma unroll 1
     for (int r2 = 0; r2 < K1; ++r2) {
         uint64_t best = 0;
-#pragma unroll 2
+#pragma unroll 8
         for (int w = e0 + lane; w < e1; w += 32) {
             const uint64_t kk = row_key(load_logit<T>(src + w), w);
             if (kk < prev && kk > best) best = kk;
