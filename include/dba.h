@@ -18,6 +18,10 @@
  *   - Logits must be finite or -inf.  NaN or +inf input is undefined behaviour of the selection
  *     (never of memory safety).
  *   - Limits: k <= 64, at most 64 constraint tokens per sentence, k*V < 2^31, V >= 1.
+ *   - Speed: the streaming row scan needs 16-byte aligned rows (base pointer and row stride) whose length in
+ *     bytes is a multiple of 16 and at most 1 MiB; other shapes are served by a plain multi-pass kernel, exact
+ *     but many times slower.  Rows in which more than 256 entries of a 44 KB stretch tie at the value of its
+ *     (k+2)-th largest entry cost an extra pass over that stretch (dba_counters reports how often).
  *
  * Slot kinds: a slot is EMPTY when its score is -inf, FINISHED when it is live and its last token is
  * eos_id, OPEN otherwise.  After dba_init (and dba_reset) slot 0 of every sentence is open with score 0
