@@ -41,6 +41,10 @@ def test_host_side_argument_checks_need_no_gpu():
     assert L.dba_workspace_bytes(C.byref(mk(logit_dtype=3)), C.byref(n)) == 1
     assert L.dba_workspace_bytes(C.byref(mk(flags=64)), C.byref(n)) == 1
     assert L.dba_workspace_bytes(None, C.byref(n)) == 1
+    assert L.dba_workspace_bytes(C.byref(mk(prune_threshold=float("nan"))), C.byref(n)) == 1
+    assert L.dba_workspace_bytes(C.byref(mk(prune_threshold=-1.0)), C.byref(n)) == 0     # <= 0: no pruning
+    assert L.dba_workspace_bytes(C.byref(mk(prune_threshold=20.0)), C.byref(n)) == 0
+    assert L.dba_counters(None, (C.c_uint32 * 4)()) == 1
     assert L.dba_status_string(0) == b"ok" and L.dba_status_string(5) == b"device-side wait timed out"
     assert L.dba_step(None, None, 0, None, None) == 1
     assert L.dba_launch_count(None) == 0
