@@ -17,7 +17,11 @@
  *   - Token ids are int32 in [0, V).  pad_id / bos_id / eos_id are the special symbols.
  *   - Logits must be finite or -inf.  NaN or +inf input is undefined behaviour of the selection
  *     (never of memory safety).
- *   - Limits: k <= 64, at most 64 constraint tokens per sentence, k*V < 2^31, V >= 1.
+ *   - Limits: k <= 64, at most 64 constraint tokens per sentence, k*V < 2^31, V >= 1.  One thread block keeps
+ *     a sentence's k*(P+2) candidates (P = phrases of the sentence that has most) and its rows' partial
+ *     lists in shared memory: every constraint set fits for k <= 40; at k = 64 sets of up to 36 phrases fit
+ *     for rows of up to 352 KB and sets of up to 12 phrases for rows of up to 1 MiB.  dba_init returns
+ *     DBA_ERR_UNSUPPORTED when the configuration does not fit.
  *   - Speed: the streaming row scan needs 16-byte aligned rows (base pointer and row stride) whose length in
  *     bytes is a multiple of 16 and at most 1 MiB; other shapes are served by a plain multi-pass kernel, exact
  *     but many times slower.  Rows in which more than 256 entries of a 44 KB stretch tie at the value of its
@@ -42,7 +46,8 @@ typedef struct dba_handle dba_handle;
 typedef enum {
     DBA_OK = 0,
     DBA_ERR_INVALID_ARG = 1,   /* null pointer, bad size, malformed constraint table, bad token id      */
-    DBA_ERR_UNSUPPORTED = 2,   /* over a documented limit (k > 64, > 64 constraint tokens, k*V >= 2^31) */
+    DBA_ERR_UNSUPPORTED = 2,   /* over a documented limit (k > 64, > 64 constraint tokens, k*V >= 2^31,
+                                  candidates beyond shared memory)                                      */
     DBA_ERR_STATE = 3,         /* step after max_steps, host-staging call without the staging flag     */
     DBA_ERR_CUDA = 4,          /* a CUDA runtime call failed                                            */
     DBA_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up (reported by dba_finalize)        */

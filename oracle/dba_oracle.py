@@ -108,7 +108,7 @@ class Sentence:
             lib().orc_set_prune(self._h, prune)
 
     def __del__(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and lib is not None:      # module globals are gone at interpreter exit
             lib().orc_destroy(self._h)
             self._h = None
 

@@ -575,14 +575,21 @@ static int pick_threads(const Dims& d, size_t smem_limit) {
 
 size_t candidates_smem_bytes(const Dims& d) { return (size_t)make_layout(d.k, d.K1, d.S, d.max_cand, 256 / 32).total; }
 
-cudaError_t configure_candidates(const Dims& d) {
+// The dynamic shared memory a block may ask for is the device's opt-in limit less what the kernel declares
+// statically.  *fits = false (and nothing configured) when even the smallest block is over it.
+cudaError_t configure_candidates(const Dims& d, bool* fits) {
     int dev = 0, lim = 0;
+    *fits = false;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&lim, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    cudaFuncAttributes fa{};
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, candidates_kernel);
     if (e != cudaSuccess) return e;
-    g_smem_limit = (size_t)lim;
+    g_smem_limit = (size_t)lim > fa.sharedSizeBytes ? (size_t)lim - fa.sharedSizeBytes : 0;
     e = cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
+    if (candidates_smem_bytes(d) > g_smem_limit) return cudaSuccess;
+    *fits = true;
     const int t = pick_threads(d, g_smem_limit);
     return cudaFuncSetAttribute(candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 make_layout(d.k, d.K1, d.S, d.max_cand, t / 32).total);

@@ -199,11 +199,9 @@ dba_status dba_init(const dba_config* cfg, void* workspace_dev, size_t workspace
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
     if (e != cudaSuccess) { delete h; return DBA_ERR_CUDA; }
     plan_segments(h->d, h->sm_count);
-    int smem_max = 0;
-    e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
-    if (e != cudaSuccess) { delete h; return DBA_ERR_CUDA; }
-    if (candidates_smem_bytes(h->d) > (size_t)smem_max) { delete h; return DBA_ERR_UNSUPPORTED; }
-    e = configure_candidates(h->d);
+    bool fits = false;
+    e = configure_candidates(h->d, &fits);
+    if (e == cudaSuccess && !fits) { delete h; return DBA_ERR_UNSUPPORTED; }
     if (e == cudaSuccess) e = configure_row_scan_tma();
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(h->cons, cons.data(), sizeof(SentCons) * cons.size(), cudaMemcpyHostToDevice, h->stream);

@@ -108,7 +108,7 @@ cudaError_t launch_finalize(const Dims& d, const Beam& beam, const int32_t* hist
 
 size_t candidates_smem_bytes(const Dims& d);
 // Opts the candidate kernel in to the dynamic shared memory it needs on the current device.
-cudaError_t configure_candidates(const Dims& d);
+cudaError_t configure_candidates(const Dims& d, bool* fits);
 
 // Chooses S and seg_len for a row of V elements when R rows are scanned (fills d.S, d.seg_len, d.K1).
 void plan_segments(Dims& d, int sm_count);

@@ -169,6 +169,13 @@ EDGE = {
     "self_overlapping_phrase": dict(B=1, k=6, V=120, steps=14, constraints=[[[8, 8, 9], [8, 9]]]),
     "big_beam":               dict(B=2, k=64, V=2048, steps=8, constraints=[[[5, 6], [7]], [[9]]], dtype="bf16"),
     "plain_normal_rows":      dict(B=2, k=7, V=900, steps=10, constraints=[[[5]], [[6, 7, 8]]], zipf=False),
+    # more sentences than the GPU holds blocks of the candidate kernel at once; constraint sets of 0-3 phrases
+    "many_sentences":         dict(B=1200, k=3, V=260, steps=6,
+                                   constraints=[[[10 + (i + j) % 50 + q for q in range(1 + (i + j) % 2)] for j in range(i % 4)]
+                                                for i in range(1200)]),
+    # the widest beam with as many one-word constraints as its candidates leave room for in shared memory
+    "widest_beam_forty_constraints": dict(B=1, k=64, V=3000, steps=10, constraints=[[[w] for w in range(100, 140)]]),
+    "beam_of_forty_most_constraints": dict(B=1, k=40, V=3000, steps=10, constraints=[[[w] for w in range(100, 164)]]),
 }
 
 
@@ -322,10 +329,16 @@ def test_argument_errors_are_reported_not_launched(dba):
     mk = lambda **kw: dba.DbaStepper(**{**dict(B=1, k=2, V=50, max_steps=3, constraints=[[[5]]]), **kw})
     for kw, code in [(dict(k=65), 2), (dict(constraints=[[[w] for w in range(4, 69)]], V=100), 2),
                      (dict(constraints=[[[2]]]), 1), (dict(constraints=[[[50]]]), 1), (dict(constraints=[[[]]]), 1),
-                     (dict(k=0), 1), (dict(V=2**31 // 2, k=2), 2), (dict(dtype=7), 1), (dict(eos=99), 1)]:
+                     (dict(k=0), 1), (dict(V=2**31 // 2, k=2), 2),
+                     (dict(k=64, V=3000, constraints=[[[w] for w in range(100, 164)]]), 2),    # candidates beyond shared memory
+                     (dict(dtype=7), 1), (dict(eos=99), 1)]:
         with pytest.raises(dba.DbaError) as e:
             mk(**kw)
         assert e.value.code == code, kw
+    ones = lambda n: [[[w] for w in range(100, 100 + n)]]
+    for kw in [dict(k=64, V=88000, constraints=ones(36)), dict(k=64, V=40000, constraints=ones(36)),
+               dict(k=64, V=262144, constraints=ones(12)), dict(k=40, V=262144, constraints=ones(64))]:          # the corners the header promises
+        mk(**kw).close()
     st = mk()
     with pytest.raises(dba.DbaError) as e:
         st.step_host(torch.zeros(2, 50), st.new_outputs(host=True))
