@@ -51,10 +51,12 @@ def assert_beam_equal(got, want, where, fields=BEAM_FIELDS + ("score",)):
                                  f"gpu    {({g: got[g][r] for g in fields})}\noracle {({g: want[g][r] for g in fields})}")
 
 
-def lockstep(wl, stepper, steps=None, threads=8, gpu_gen=None, lse_tol=1e-5, flags=0, prune=0.0):
+def lockstep(wl, stepper, steps=None, threads=8, gpu_gen=None, lse_tol=1e-5, flags=0, prune=0.0, row_pad=0):
     """Closed loop with the oracle's row normalisers handed to the CUDA step (the direction oracle -> GPU),
     so that both rank the same fp32 score matrix: every selection output must then match bit for bit at
-    every step, and the normalisers the GPU computes itself must agree within lse_tol."""
+    every step, and the normalisers the GPU computes itself must agree within lse_tol.
+    row_pad > 0: the device rows are row_pad elements apart beyond their length, the gaps filled with a value
+    larger than any logit (a read past the end of a row would win every selection)."""
     import torch
     steps = wl.steps if steps is None else steps
     orc = O.Batch(wl.k, wl.V, steps, wl.constraints, flags=flags & 3, threads=threads, prune=prune)
@@ -69,6 +71,10 @@ def lockstep(wl, stepper, steps=None, threads=8, gpu_gen=None, lse_tol=1e-5, fla
         else:
             x_np = host_gen.step_logits(t, ob["token"], ob["met_mask"])
             x_dev = to_device_logits(x_np, wl)
+        if row_pad:
+            wide = torch.full((x_dev.shape[0], wl.V + row_pad), 3.0e4, dtype=x_dev.dtype, device=x_dev.device)
+            wide[:, :wl.V] = x_dev
+            x_dev = wide[:, :wl.V]
         open_rows = np.isfinite(ob["score"]) & (ob["token"] != 2)
         lse_o = orc.step(x_np)
         out = stepper.step(x_dev, row_lse_in=torch.from_numpy(lse_o).cuda())

@@ -169,6 +169,9 @@ EDGE = {
     "self_overlapping_phrase": dict(B=1, k=6, V=120, steps=14, constraints=[[[8, 8, 9], [8, 9]]]),
     "big_beam":               dict(B=2, k=64, V=2048, steps=8, constraints=[[[5, 6], [7]], [[9]]], dtype="bf16"),
     "plain_normal_rows":      dict(B=2, k=7, V=900, steps=10, constraints=[[[5]], [[6, 7, 8]]], zipf=False),
+    # fewer words than beam slots: rows shorter than the k+2 entries the scan keeps, beams that cannot fill
+    "vocab_smaller_than_beam": dict(B=2, k=8, V=8, steps=8, constraints=[[[3]], [[4, 5]]]),
+    "vocab_smaller_than_beam_bf16": dict(B=2, k=12, V=9, steps=8, constraints=[[[3]], [[4, 5], [6]]], dtype="bf16"),
     # more sentences than the GPU holds blocks of the candidate kernel at once; constraint sets of 0-3 phrases
     "many_sentences":         dict(B=1200, k=3, V=260, steps=6,
                                    constraints=[[[10 + (i + j) % 50 + q for q in range(1 + (i + j) % 2)] for j in range(i % 4)]
@@ -185,6 +188,16 @@ def test_step_parity_edge_cases(dba, case):
     wl = _custom(case, **p)
     st = _stepper(dba, wl)
     orc, worst = lockstep(wl, st)
+    assert_finalize_equal(st, orc)
+
+
+@pytest.mark.parametrize("dtype,V,pad", [("f32", 4096, 64), ("bf16", 24576, 8), ("f32", 1003, 5), ("bf16", 4096, 3)])
+def test_rows_further_apart_than_their_length(dba, dtype, V, pad):
+    """row_stride_elems > V, with the gaps holding values above every logit: aligned strides take the streaming
+    scan, the others the plain one; neither the scan nor the progress-token look-ups may read a gap."""
+    wl = _custom("padded", B=3, k=5, V=V, steps=10, constraints=[[[5, 6]], [[7], [8, 9, 10]], []], dtype=dtype)
+    st = _stepper(dba, wl)
+    orc, worst = lockstep(wl, st, row_pad=pad)
     assert_finalize_equal(st, orc)
 
 
