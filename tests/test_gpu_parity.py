@@ -176,6 +176,10 @@ EDGE = {
     "many_sentences":         dict(B=1200, k=3, V=260, steps=6,
                                    constraints=[[[10 + (i + j) % 50 + q for q in range(1 + (i + j) % 2)] for j in range(i % 4)]
                                                 for i in range(1200)]),
+    "eighty_thousand_rows":   dict(B=4096, k=20, V=256, steps=3, constraints=[[[10 + i % 100]] * (i % 3) for i in range(4096)]),
+    # steps go on long after every hypothesis has ended (no open row is left to scan)
+    "steps_after_the_end":    dict(B=1, k=3, V=100, steps=40, constraints=[[[5]]]),
+    "steps_after_one_sentence_ended": dict(B=2, k=3, V=100, steps=40, constraints=[[[5]], [[6, 7]]]),
     # the widest beam with as many one-word constraints as its candidates leave room for in shared memory
     "widest_beam_forty_constraints": dict(B=1, k=64, V=3000, steps=10, constraints=[[[w] for w in range(100, 140)]]),
     "beam_of_forty_most_constraints": dict(B=1, k=40, V=3000, steps=10, constraints=[[[w] for w in range(100, 164)]]),
@@ -320,6 +324,10 @@ def test_step_host_equals_step_and_reset_replays(dba):
         x = gen.step_logits(t, tok, mask)
         ga = gpu_beam(a.step(to_device_logits(x, wl)))
         xh = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory()
+        if t % 2:                      # host rows further apart than their length, the gaps above every logit
+            wide = torch.full((wl.R, wl.V + 24), 3.0e4, dtype=torch.bfloat16).pin_memory()
+            wide[:, :wl.V] = xh
+            xh = wide[:, :wl.V]
         b.step_host(xh, host_out)
         gb = {f: host_out[f].numpy().copy() for f in host_out}
         gb["met_mask"] = gb["met_mask"].view(np.uint64)
