@@ -72,7 +72,7 @@ def _rows(kind, R, V, rng):
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("kind", ["normal", "ascending", "descending", "constant", "quantised", "holes", "signed_zero"])
 @pytest.mark.parametrize("V,n_top", [(1, 3), (7, 7), (1000, 7), (4099, 22), (32000, 12), (64000, 22), (20011, 66),
-                                      (24576, 12), (150000, 22), (262144, 7)])
+                                      (24576, 12), (150000, 22), (262144, 7), (1000003, 22), (1048576, 12)])
 def test_row_scan_matches_oracle(dba, dtype, kind, V, n_top):
     from synth_inputs.logits import to_bf16_bits
     rng = np.random.default_rng(V + n_top)
