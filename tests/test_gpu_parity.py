@@ -150,6 +150,21 @@ def test_serving_full_size_free_run_against_sampled_oracle(dba):
     assert left <= 1 and compared >= 4 * steps
 
 
+@pytest.mark.parametrize("dtype,B,V", [("f32", 210, 262144), ("bf16", 212, 524288)])
+def test_logit_matrices_beyond_four_gigabytes(dba, dtype, B, V):
+    """Rows of 1 MiB, more than 4096 of them: the byte offsets of the last sentences' rows do not fit 32 bits
+    (f32: 4.4 GB; bf16: 4.4 GB as well, 2.2e9 elements, more than 2^31).  Free-running; the oracle follows the first, a middle and the last sentences."""
+    from synth_inputs.gpu import GpuLogitStream
+    from tests.parity import free_run
+    wl = make_workload("scaling", C=5, B=B, V=V, dtype=dtype)
+    assert wl.R * wl.V * (4 if dtype == "f32" else 2) > 2**32
+    st = _stepper(dba, wl)
+    steps = 5
+    sample = [0, B // 2, B - 5, B - 1]
+    compared, left = free_run(wl, st, sample, steps, GpuLogitStream(wl))
+    assert left <= 1 and compared >= 3 * steps
+
+
 # ------------------------------------------------------------------------------------------ edge cases
 def _custom(name, B, k, V, steps, constraints, dtype="f32", zipf=True):
     from synth_inputs.configs import Workload
