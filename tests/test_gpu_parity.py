@@ -220,6 +220,30 @@ def test_rows_further_apart_than_their_length(dba, dtype, V, pad):
     assert_finalize_equal(st, orc)
 
 
+def test_special_symbols_elsewhere_in_the_vocabulary(dba):
+    """pad, bos and eos are configuration, not 0, 1, 2: here they sit at the end and in the middle of the
+    vocabulary (the stream's columns 0, 1, 2 are moved there) and 0, 1, 2 are ordinary, constrained words."""
+    V, k, B, steps = 1200, 6, 3, 16
+    pad, bos, eos = 1199, 640, 77
+    wl = _custom("ids", B=B, k=k, V=V, steps=steps, constraints=[[[5, 6]], [[0], [2, 1]], []], dtype="bf16")
+    perm = np.arange(V); perm[[0, pad]] = [pad, 0]; perm[[1, bos]] = [bos, 1]; perm[[2, eos]] = [eos, 2]
+    st = dba.DbaStepper(B, k, V, steps, constraints=wl.constraints, dtype=dba.BF16, pad=pad, bos=bos, eos=eos)
+    orc = O.Batch(k, V, steps, wl.constraints, pad=pad, bos=bos, eos=eos, threads=1)
+    gen = LogitStream(wl)
+    for t in range(steps):
+        ob = orc.beam()
+        x = np.ascontiguousarray(gen.step_logits(t, ob["token"], ob["met_mask"])[:, perm])
+        lse_o = orc.step(x)
+        out = st.step(to_device_logits(x, wl), row_lse_in=torch.from_numpy(lse_o).cuda())
+        assert_beam_equal(gpu_beam(out), orc.beam(), f"step {t}")
+    tokens, length, score, flags = st.finalize()
+    want = orc.finalize()
+    assert all(done for _, _, done in want)
+    for b, (toks, sc, done) in enumerate(want):
+        assert tokens[b, :length[b]].tolist() == toks and toks[-1] == eos and (tokens[b, length[b]:] == pad).all()
+        assert score[b] == np.float32(sc) and flags[b] & 1
+
+
 @pytest.mark.parametrize("name,kw,theta", [("tiny", {}, 3.0), ("ragged", dict(B=6, V=4096, steps=40), 20.0),
                                            ("ragged", dict(B=6, V=4096, steps=40), 2.0),
                                            ("serving", dict(B=3, V=8192, steps=60), 5.0)])
