@@ -590,9 +590,9 @@ cudaError_t configure_candidates(const Dims& d, bool* fits) {
     if (e != cudaSuccess) return e;
     if (candidates_smem_bytes(d) > g_smem_limit) return cudaSuccess;
     *fits = true;
-    const int t = pick_threads(d, g_smem_limit);
-    return cudaFuncSetAttribute(candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                make_layout(d.k, d.K1, d.S, d.max_cand, t / 32).total);
+    // The attribute belongs to the kernel, not to a handle: it is raised to the most any shape may ask for, so
+    // that handles of different shapes can be alive together.
+    return cudaFuncSetAttribute(candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g_smem_limit);
 }
 
 cudaError_t launch_candidates(const void* logits, int64_t stride, const Dims& d, const SentCons* cons,

@@ -220,6 +220,24 @@ def test_rows_further_apart_than_their_length(dba, dtype, V, pad):
     assert_finalize_equal(st, orc)
 
 
+def test_handles_of_different_shapes_alive_together(dba):
+    """A handle that needs nearly all the shared memory of a block keeps working after a small one was made
+    (what a launch may ask for is a property of the kernel, shared by all handles), steps interleaved."""
+    big = _custom("big", **EDGE["widest_beam_forty_constraints"])
+    small = _custom("small", **EDGE["beam_of_one"])
+    st_big = _stepper(dba, big)
+    st_small = _stepper(dba, small)                 # initialised second: must not lower the first one's limit
+    orcs = {n: O.Batch(w.k, w.V, w.steps, w.constraints, threads=1) for n, w in (("big", big), ("small", small))}
+    gens = {"big": LogitStream(big), "small": LogitStream(small)}
+    for t in range(8):
+        for n, w, st in (("big", big, st_big), ("small", small, st_small)):
+            ob = orcs[n].beam()
+            x = gens[n].step_logits(t, ob["token"], ob["met_mask"])
+            lse_o = orcs[n].step(x)
+            out = st.step(to_device_logits(x, w), row_lse_in=torch.from_numpy(lse_o).cuda())
+            assert_beam_equal(gpu_beam(out), orcs[n].beam(), f"{n} step {t}")
+
+
 def test_special_symbols_elsewhere_in_the_vocabulary(dba):
     """pad, bos and eos are configuration, not 0, 1, 2: here they sit at the end and in the middle of the
     vocabulary (the stream's columns 0, 1, 2 are moved there) and 0, 1, 2 are ordinary, constrained words."""
