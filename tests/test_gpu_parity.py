@@ -184,6 +184,10 @@ EDGE = {
     "self_overlapping_phrase": dict(B=1, k=6, V=120, steps=14, constraints=[[[8, 8, 9], [8, 9]]]),
     "big_beam":               dict(B=2, k=64, V=2048, steps=8, constraints=[[[5, 6], [7]], [[9]]], dtype="bf16"),
     "plain_normal_rows":      dict(B=2, k=7, V=900, steps=10, constraints=[[[5]], [[6, 7, 8]]], zipf=False),
+    # k + 2 = 32 entries per row is the widest list the candidate kernel merges in registers; 33 takes the other way
+    "beam_of_thirty":         dict(B=2, k=30, V=30000, steps=8, constraints=[[[5, 6], [7]], [[9], [10], [11, 12, 13]]], dtype="bf16"),
+    "beam_of_thirty_one":     dict(B=2, k=31, V=30000, steps=8, constraints=[[[5, 6], [7]], [[9], [10], [11, 12, 13]]], dtype="bf16"),
+    "widest_beam_long_rows":  dict(B=2, k=64, V=64000, steps=6, constraints=[[[5, 6], [7]], [[9]]], dtype="bf16"),
     # fewer words than beam slots: rows shorter than the k+2 entries the scan keeps, beams that cannot fill
     "vocab_smaller_than_beam": dict(B=2, k=8, V=8, steps=8, constraints=[[[3]], [[4, 5]]]),
     "vocab_smaller_than_beam_bf16": dict(B=2, k=12, V=9, steps=8, constraints=[[[3]], [[4, 5], [6]]], dtype="bf16"),
@@ -236,6 +240,26 @@ def test_handles_of_different_shapes_alive_together(dba):
             lse_o = orcs[n].step(x)
             out = st.step(to_device_logits(x, w), row_lse_in=torch.from_numpy(lse_o).cuda())
             assert_beam_equal(gpu_beam(out), orcs[n].beam(), f"{n} step {t}")
+
+
+def test_steps_on_a_stream_of_the_callers(dba):
+    """Everything the library enqueues goes to the stream given at initialisation (here not the default one):
+    inputs are made ready before, outputs read after a synchronisation of that stream alone."""
+    wl = make_workload("ragged", B=5, V=4096, steps=20)
+    s = torch.cuda.Stream()
+    st = dba.DbaStepper(wl.B, wl.k, wl.V, wl.steps, constraints=wl.constraints, dtype=dba.BF16, stream=s)
+    orc = O.Batch(wl.k, wl.V, wl.steps, wl.constraints, threads=1)
+    gen = LogitStream(wl)
+    for t in range(wl.steps):
+        ob = orc.beam()
+        x = gen.step_logits(t, ob["token"], ob["met_mask"])
+        lse_o = orc.step(x)
+        x_dev, lse_dev = to_device_logits(x, wl), torch.from_numpy(lse_o).cuda()
+        torch.cuda.current_stream().synchronize()
+        out = st.step(x_dev, row_lse_in=lse_dev)
+        s.synchronize()
+        assert_beam_equal(gpu_beam(out), orc.beam(), f"step {t}")
+    assert_finalize_equal(st, orc)
 
 
 def test_special_symbols_elsewhere_in_the_vocabulary(dba):
