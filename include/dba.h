@@ -15,8 +15,7 @@
  *   - dba_step only enqueues work on the stream given to dba_init and does not synchronise.
  *   - Row r = b*k + h of any [B*k, ...] array belongs to beam slot h of sentence b.
  *   - Token ids are int32 in [0, V).  pad_id / bos_id / eos_id are the special symbols.
- *   - Logits must be finite or -inf.  NaN or +inf input is undefined behaviour of the selection
- *     (never of memory safety).
+ *   - Logits must be finite or -inf.  With NaN or +inf in a row the selection is unspecified.
  *   - Limits: k <= 64, at most 64 constraint tokens per sentence, k*V < 2^31, V >= 1.  One thread block keeps
  *     a sentence's k*(P+2) candidates (P = phrases of the sentence that has most) and its rows' partial
  *     lists in shared memory: every constraint set fits for k <= 40; at k = 64 sets of up to 36 phrases fit

@@ -55,7 +55,7 @@ __global__ void finalize_kernel(Dims d, Beam beam, const int32_t* __restrict__ h
     int slot = pick;
     for (int t = steps - 1; t >= 0; --t) {        // walk the back-pointers, writing tokens in place
         out[t] = hist_tok[(int64_t)t * d.R + r0 + slot];
-        slot = hist_bp[(int64_t)t * d.R + r0 + slot];
+        slot = min(max(hist_bp[(int64_t)t * d.R + r0 + slot], 0), k - 1);   // a record is a slot number; never trusted as an index
     }
     int n = 0;
     while (n < steps) { ++n; if (out[n - 1] == d.eos_id) break; }
