@@ -21,6 +21,10 @@
  *     lists in shared memory: every constraint set fits for k <= 40; at k = 64 sets of up to 36 phrases fit
  *     for rows of up to 352 KB and sets of up to 12 phrases for rows of up to 1 MiB.  dba_init returns
  *     DBA_ERR_UNSUPPORTED when the configuration does not fit.
+ *   - Threads: calls on one handle must not overlap, nor may two dba_init calls (the kernels' launch limits
+ *     are set there, once per process and device); different handles may otherwise be used from different
+ *     host threads.  A handle belongs to the device that was current in dba_init; make it current again for
+ *     every call on the handle.
  *   - Speed: the streaming row scan needs 16-byte aligned rows (base pointer and row stride) whose length in
  *     bytes is a multiple of 16 and at most 1 MiB; other shapes are served by a plain multi-pass kernel, exact
  *     but many times slower.  Rows in which more than 256 entries of a 44 KB stretch tie at the value of its
