@@ -365,8 +365,10 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
             uint4 v[kVecsPerLane];
             typename Vec<T>::Max pmax[kPairs];
             uint32_t key = 0;                      // below the key of every value, -inf included
+            // A warp without a chunk in this item waits for the copy all the same: it must not run ahead and sign
+            // the buffer off (`loaded`) for this use while a slower warp has yet to do so for the previous one.
+            if (!mbar_wait_warp(smem_u32(&sm.full[slot]), it.slot_phase(), abort_flag)) break;
             if (nvec > 0) {
-                if (!mbar_wait_warp(smem_u32(&sm.full[slot]), it.slot_phase(), abort_flag)) break;
                 const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[slot]) + chunk * kChunkVecs + lane;
                 if (nvec >= kChunkVecs) {
 #pragma unroll
