@@ -97,6 +97,36 @@ def test_row_scan_matches_oracle(dba, dtype, kind, V, n_top):
         assert np.array_equal(val[r], wv)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_repeated_scans_of_the_same_rows_agree(dba, dtype):
+    """The streaming scan's warps hand work to one another through barriers; a mistake in that hand-over shows
+    as a result that changes from launch to launch.  30 launches over the same 3000 benchmark-shaped rows must
+    give the same bits, and sampled rows must match the oracle."""
+    from synth_inputs.logits import to_bf16_bits
+    R, V, n_top = 3000, 64000, 22
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    mu = -1.1 * torch.log(torch.randperm(V, device="cuda", generator=g).float() + 1)
+    x = torch.randn(R, V, device="cuda", generator=g) + mu
+    if dtype == "bf16":
+        x = x.to(torch.bfloat16)
+    first = None
+    for it in range(30):
+        lse, val, idx = dba.row_scan(x, n_top)
+        got = (lse.clone(), val.clone(), idx.clone())
+        if first is None:
+            first = got
+        else:
+            for a, b, what in zip(got, first, ("lse", "values", "indices")):
+                assert torch.equal(a, b), f"launch {it}: {what} differ from the first launch in {int((a != b).any(-1).sum() if a.dim() > 1 else (a != b).sum())} rows"
+    lse, val, idx = (t.cpu().numpy() for t in first)
+    for r in (0, 1, 1499, 2998, 2999):
+        row = x[r].float().cpu().numpy()
+        row_in = to_bf16_bits(row) if dtype == "bf16" else row
+        wv, wi = O.row_top(row_in, n_top)
+        assert np.array_equal(idx[r], wi) and np.array_equal(val[r], wv)
+        assert abs(float(lse[r]) - O.row_lse(row_in)) <= 1e-5
+
+
 # ------------------------------------------------------------------------------------------ whole step
 def test_step_parity_tiny(dba):
     wl = make_workload("tiny")
