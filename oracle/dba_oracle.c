@@ -14,20 +14,28 @@
  * status (what the CPU tests tie each function to, other than itself):
  *   orc_row_lse        pinned   closed forms (constant, two-value, geometric rows), shift invariance
  *   orc_row_top        pinned   equals a stable descending sort of the row
+ *   orc_project        pinned   one-hot hidden state returns a row of the embedding; constant hidden state
+ *                               returns scaled row sums; small integers give exact integer inner products
  *   step at C = 0      pinned   equals Algorithm 1's ARGMAX_K over the k x V matrix (full sort)
  *   candidate set      pinned   brute force by predicate over every (h, w) cell on small V, k
  *   orc_add            pinned   hand traces of Section 3.1's unwinding text; substring semantics on
- *                               non-overlapping phrases; exhaustive search regime
+ *                               non-overlapping phrases; exhaustive search regime;
+ *                               parity unpinned: continuation before opening, first matching constraint
+ *                               (conventions; tests/golden/add_masks.txt holds them as such)
  *   orc_allocate       pinned   Fig. 1 / Fig. 2 captions (k = 5, four constraints), sum = min(k, #cand),
- *                               alloc <= count, C >= k;
- *                               parity unpinned: the exact split among several deficit banks (the
- *                               paper only outlines the procedure and the figure that shows one is lost)
+ *                               alloc <= count, C >= k; nearest-bank-first and moving outward (Section 3.2's
+ *                               adjustment sentence) by hand-derived allocations without ties;
+ *                               parity unpinned: which of two equally near banks is served first and the
+ *                               order in which overfilled banks act (the paper only outlines the procedure
+ *                               and the figure that shows one is lost)
  *   finishing          pinned   every completed output holds all constraints; exhaustive regime
  *                               equals brute force over all sequences
  *   pruning, stopping  pinned   closed form on a two-word vocabulary (two scores exactly theta' apart: kept iff
  *                               theta' <= threshold), the best completed hypothesis is never removed, an
  *                               infinite threshold changes nothing, stop bits on hand-built beams;
- *                               parity unpinned: which score is compared (READING below)
+ *                               the other reading (normalised completed scores, ORC_FLAG_PRUNE_NORM) by a
+ *                               hand-built beam on which the two readings remove different hypotheses;
+ *                               parity unpinned: which of the two readings the paper means
  *   conventions        parity unpinned: finished hypotheses staying on the beam with a frozen
  *                               score, empty slots, global order of the new beam, length counted
  *                               with the end token (READINGS below)
@@ -40,7 +48,7 @@
 #define ORC_MAX_C 64
 
 enum { ORC_F32 = 0, ORC_BF16 = 1 };
-enum { ORC_FLAG_ADJUST_OFF = 1u, ORC_FLAG_LENGTH_NORM = 2u };
+enum { ORC_FLAG_ADJUST_OFF = 1u, ORC_FLAG_LENGTH_NORM = 2u, ORC_FLAG_PRUNE_NORM = 8u };
 
 typedef struct {
     int h, w;          /* coordinates in the k x V matrix (Section 3.1 names a candidate by its cell) */
@@ -94,6 +102,24 @@ double orc_row_lse(const void *row, int dtype, int V)
     double s = 0.0;
     for (int w = 0; w < V; ++w) s += exp((double)widen(row, dtype, w) - m);
     return m + log(s);
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Section 2, DECODER-STEP's last stage (Algorithm 1 line 4 produces the k x |V_T| matrix): the model output
+ * for hypothesis r and word w is the inner product of the decoder's final hidden state h_r with the
+ * output embedding E_w.  Plain triple loop, bf16 inputs widened exactly, accumulation in double in
+ * index order, one rounding to fp32 at the end.
+ *   hidden: [R, d] bf16 bits;  embed: [V, d] bf16 bits;  logits_out: [R, V] fp32.
+ * ------------------------------------------------------------------------------------------ */
+void orc_project(const uint16_t *hidden, const uint16_t *embed, int R, int V, int d, float *logits_out)
+{
+    for (int r = 0; r < R; ++r)
+        for (int w = 0; w < V; ++w) {
+            double acc = 0.0;
+            for (int j = 0; j < d; ++j)
+                acc += (double)widen(hidden + (size_t)r * d, ORC_BF16, j) * (double)widen(embed + (size_t)w * d, ORC_BF16, j);
+            logits_out[(size_t)r * V + w] = (float)acc;
+        }
 }
 
 /* ------------------------------------------------------------------------------------------
@@ -435,18 +461,30 @@ int orc_step(orc_sentence *s, const void *logits, int dtype, long row_stride, fl
     /* Section 4 (and Section 6.3): threshold pruning of the beam.  A hypothesis whose log-probability is not
        within the threshold of the best completed hypothesis is removed, whether it is itself complete or not.
        READING: both sides of the comparison are cumulative log-probabilities (the scores the beam is ordered
-       by); a removed hypothesis leaves an empty slot; the beam is in decreasing order, so they are its tail. */
+       by); a removed hypothesis leaves an empty slot and the hypotheses behind it move up.
+       OTHER READING (ORC_FLAG_PRUNE_NORM): Section 4 first says that completed hypotheses are normalised
+       (cumulative score divided by the number of words) and then states the pruning rule, so the value a
+       completed hypothesis enters the comparison with is its normalised score (on both sides: as the
+       reference, and when it is itself tested); a hypothesis that is not completed enters with its cumulative
+       score.  The beam stays ordered by cumulative score. */
     if (s->prune > 0) {
+        float *val = (float *)malloc(sizeof(float) * (nkept + 1));
+        for (int i = 0; i < nkept; ++i) {
+            val[i] = kept[i].score;
+            if ((s->flags & ORC_FLAG_PRUNE_NORM) && kept[i].w == s->eos && kept[i].len > 0)
+                val[i] = kept[i].score / (float)kept[i].len;
+        }
         float best = -INFINITY;
         for (int i = 0; i < nkept; ++i)
-            if (kept[i].w == s->eos && kept[i].score > best) best = kept[i].score;
+            if (kept[i].w == s->eos && val[i] > best) best = val[i];
         if (best != -INFINITY) {
             volatile float cut = best - s->prune;
             int n = 0;
             for (int i = 0; i < nkept; ++i)
-                if (!(kept[i].score < cut)) kept[n++] = kept[i];
+                if (!(val[i] < cut)) kept[n++] = kept[i];
             nkept = n;
         }
+        free(val);
     }
 
     int *hb = s->hist_bp + (size_t)s->t * k, *ht = s->hist_tok + (size_t)s->t * k;

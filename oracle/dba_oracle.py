@@ -17,7 +17,7 @@ _SRC = os.path.join(_HERE, "dba_oracle.c")
 _LIB = os.path.join(_HERE, "libdba_oracle.so")
 
 F32, BF16 = 0, 1
-FLAG_ADJUST_OFF, FLAG_LENGTH_NORM = 1, 2
+FLAG_ADJUST_OFF, FLAG_LENGTH_NORM, FLAG_PRUNE_NORM = 1, 2, 8
 
 _lib = None
 
@@ -39,6 +39,8 @@ def lib():
         L.orc_row_lse.restype = C.c_double
         L.orc_row_lse.argtypes = [C.c_void_p, C.c_int, C.c_int]
         L.orc_row_top.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, f32p, i32p]
+        L.orc_project.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, f32p]
+        L.orc_project.restype = None
         L.orc_create.restype = C.c_void_p
         L.orc_create.argtypes = [C.c_int] * 6 + [C.c_uint, C.c_int, i32p, i32p]
         L.orc_destroy.argtypes = [C.c_void_p]
@@ -80,6 +82,18 @@ def row_top(row: np.ndarray, n: int):
     val = np.zeros(n, np.float32); idx = np.zeros(n, np.int32)
     lib().orc_row_top(row.ctypes.data, dt, row.size, n, _p(val, C.c_float), _p(idx, C.c_int32))
     return val, idx
+
+
+def project(hidden_bits: np.ndarray, embed_bits: np.ndarray) -> np.ndarray:
+    """Output projection: logits[r, w] = <hidden[r], embed[w]> (uint16 arrays of bf16 bits, [R, d] and [V, d]);
+    double accumulation, rounded once to fp32."""
+    hidden_bits = np.ascontiguousarray(hidden_bits); embed_bits = np.ascontiguousarray(embed_bits)
+    assert hidden_bits.dtype == np.uint16 and embed_bits.dtype == np.uint16 and hidden_bits.shape[1] == embed_bits.shape[1]
+    R, d = hidden_bits.shape
+    V = embed_bits.shape[0]
+    out = np.zeros((R, V), np.float32)
+    lib().orc_project(hidden_bits.ctypes.data, embed_bits.ctypes.data, R, V, d, _p(out, C.c_float))
+    return out
 
 
 def allocate(k: int, n, flags: int = 0) -> np.ndarray:

@@ -75,6 +75,26 @@ def test_add_hand_traces(golden_dir):
     assert n >= 10
 
 
+def test_add_marks_the_positions_the_conventions_name(golden_dir):
+    """Which positions are marked (tests/golden/add_masks.txt): continuation of the begun phrase wins over opening
+    another constraint; of several unmet constraints opening with the token the first in order is marked."""
+    n = 0
+    for line in open(os.path.join(golden_dir, "add_masks.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        ph, toks, want = [f.strip() for f in line.split(";")]
+        phrases = [[int(t) for t in p.split()] for p in ph.split("|")]
+        s = O.Sentence(2, 64, 4, phrases)
+        mask, active = 0, -1
+        for w in toks.split():
+            mask, active = s.add(mask, active, int(w))
+        want_mask = 0 if want == "-" else sum(1 << int(t) for t in want.split())
+        assert mask == want_mask, (line, bin(mask))
+        n += 1
+    assert n >= 8
+
+
 def _phrase_bits(phrases):
     pos, out = 0, []
     for p in phrases:
@@ -167,7 +187,7 @@ def test_allocation_figure_captions(golden_dir):
             elif e != "*":
                 assert a == int(e)
         rows += 1
-    assert rows >= 6
+    assert rows >= 13
 
 
 def test_allocation_base_share_when_every_bank_is_full():
@@ -472,6 +492,34 @@ def test_pruning_removes_completed_hypotheses_too_and_never_the_best_completed_o
     assert u.beam()["score"][3] == np.float32(-30.0) and u.beam()["token"][3] == 2
 
 
+def test_pruning_by_normalised_completed_scores_removes_what_the_hand_calculation_says():
+    """Section 4 normalises completed hypotheses (score / number of words) before it states the pruning rule.
+    Under that reading (ORC_FLAG_PRUNE_NORM) a beam of two completed hypotheses, A (-6 over 3 words: -2 per word)
+    and B (-5 over 1 word), and two open ones whose only continuation has probability 1 (C at -3.5, D at -4.5)
+    with threshold 2 keeps what is within 2 of A's -2: A (-2) and C (-3.5); B (-5) and D (-4.5) go.  Under the
+    default reading the reference is B's -5 and all four stay (all >= -7)."""
+    k, V = 4, 4
+    x = np.full((k, V), NEG, np.float32); x[2, 3] = 0.0; x[3, 3] = 0.0       # open rows: one word, probability 1
+    beam = ([-5.0, -6.0, -3.5, -4.5], [2, 2, 3, 3], [0] * 4, [-1] * 4, [1, 3, 2, 2])
+    s = O.Sentence(k, V, 3, [], flags=O.FLAG_PRUNE_NORM, prune=2.0)
+    s.set_beam(*beam)
+    s.step(x)
+    bm = s.beam()
+    # the beam stays in order of cumulative score: C (-3.5, from slot 2) before A (-6, from slot 1)
+    assert bm["score"][:2].tolist() == [-3.5, -6.0] and bm["backptr"][:2].tolist() == [2, 1]
+    assert bm["token"][:2].tolist() == [3, 2] and np.isinf(bm["score"][2:]).all()
+    u = O.Sentence(k, V, 3, [], prune=2.0)
+    u.set_beam(*beam)
+    u.step(x)
+    bu = u.beam()
+    assert bu["score"].tolist() == [-3.5, -4.5, -5.0, -6.0] and bu["backptr"].tolist() == [2, 3, 0, 1]
+    # a threshold that reaches everything: the two readings agree again
+    w = O.Sentence(k, V, 3, [], flags=O.FLAG_PRUNE_NORM, prune=10.0)
+    w.set_beam(*beam)
+    w.step(x)
+    assert np.array_equal(w.beam()["score"], bu["score"])
+
+
 def test_stop_bit_zero_needs_every_hypothesis_on_the_beam_completed():
     s = O.Sentence(3, 5, 4, [])
     s.set_beam([-1.0, -2.0, NEG], [2, 2, 0], [0] * 3, [-1] * 3, [2, 2, 0])
@@ -505,3 +553,32 @@ def test_a_huge_threshold_changes_nothing_and_survivors_are_always_within_the_th
             pruned_something |= live.sum() < np.isfinite(ba["score"]).sum()
         assert (np.diff(live.astype(int)) <= 0).all()
     assert pruned_something
+
+
+# ------------------------------------------------------------------------------------------ output projection
+def _bf16(x):
+    from synth_inputs.logits import to_bf16_bits
+    return to_bf16_bits(np.ascontiguousarray(x, np.float32))
+
+
+def test_projection_closed_forms():
+    """Section 2: the score matrix is the hidden states times the output embedding.  A one-hot hidden state
+    picks a column of the embedding; a constant one gives scaled row sums; small integers multiply exactly; a
+    transposed operand or a dropped term fails one of these."""
+    from synth_inputs.logits import bf16_bits_to_f32
+    rng = np.random.default_rng(11)
+    V, d = 37, 24
+    E = rng.normal(0, 1, (V, d)).astype(np.float32)
+    Eb = _bf16(E); Ef = bf16_bits_to_f32(Eb).astype(np.float64)
+    H = np.zeros((d, d), np.float32); H[np.arange(d), np.arange(d)] = 1.0          # row j is the j-th unit vector
+    got = O.project(_bf16(H), Eb)
+    assert got.shape == (d, V) and np.array_equal(got, Ef.T.astype(np.float32))
+    H = np.full((2, d), 0.5, np.float32); H[1] = -2.0
+    got = O.project(_bf16(H), Eb)
+    assert np.array_equal(got[0], (0.5 * Ef.sum(1)).astype(np.float32))
+    assert np.array_equal(got[1], (-2.0 * Ef.sum(1)).astype(np.float32))
+    Hi = rng.integers(-8, 9, (5, d)).astype(np.float32); Ei = rng.integers(-8, 9, (V, d)).astype(np.float32)
+    got = O.project(_bf16(Hi), _bf16(Ei))
+    assert np.array_equal(got, (Hi.astype(np.int64) @ Ei.astype(np.int64).T).astype(np.float32))
+    # not symmetric in its operands: the shapes alone catch a transposition
+    assert O.project(_bf16(Hi[:3]), _bf16(Ei)).shape == (3, V)
