@@ -21,10 +21,10 @@
  *     lists in shared memory: every constraint set fits for k <= 40; at k = 64 sets of up to 36 phrases fit
  *     for rows of up to 352 KB and sets of up to 12 phrases for rows of up to 1 MiB.  dba_init returns
  *     DBA_ERR_UNSUPPORTED when the configuration does not fit.
- *   - Threads: calls on one handle must not overlap, nor may two dba_init calls (the kernels' launch limits
- *     are set there, once per process and device); different handles may otherwise be used from different
- *     host threads.  A handle belongs to the device that was current in dba_init; make it current again for
- *     every call on the handle.
+ *   - Threads: calls on one handle must not overlap, nor may two dba_init calls (the kernels' shared-memory
+ *     limits are raised there, once per process and device); different handles may otherwise be used from
+ *     different host threads.  A handle belongs to the device that was current in dba_init; make it current
+ *     again for every call on the handle.
  *   - Speed: the streaming row scan needs 16-byte aligned rows (base pointer and row stride) whose length in
  *     bytes is a multiple of 16 and at most 1 MiB; other shapes are served by a plain multi-pass kernel, exact
  *     but many times slower.  Rows in which more than 256 entries of a 44 KB stretch tie at the value of its
@@ -62,7 +62,10 @@ typedef enum { DBA_F32 = 0, DBA_BF16 = 1 } dba_dtype;
 enum {
     DBA_FLAG_ADJUST_OFF   = 1u,  /* Section 5 (grid-beam-search simulation): no bank adjustment        */
     DBA_FLAG_LENGTH_NORM  = 2u,  /* Section 4: dba_finalize ranks completed hypotheses by score/length  */
-    DBA_FLAG_HOST_STAGING = 4u   /* reserve workspace for dba_step_host                                 */
+    DBA_FLAG_HOST_STAGING = 4u,  /* reserve workspace for dba_step_host                                 */
+    DBA_FLAG_PRUNE_NORMALISED = 8u, /* Section 4, read the other way: the threshold pruning compares completed
+                                    hypotheses by score/length (see prune_threshold)                    */
+    DBA_FLAG_FUSED_PROJECTION = 16u /* reserve workspace for dba_step_fused (needs k <= 30)              */
 };
 
 /* Bits of dba_step_out.stop (Section 4's stopping rule; Section 6.4's early stopping). */
@@ -87,7 +90,12 @@ typedef struct {
     const int32_t* tok;                /* [sum]  token ids in [0, V), none of pad/bos/eos                 */
     float prune_threshold;             /* Section 4: > 0 removes, after every step, the hypotheses (completed or
                                           not) whose score is more than this below the best completed
-                                          hypothesis on the beam (the paper uses 20); <= 0: no pruning       */
+                                          hypothesis on the beam (the paper uses 20); <= 0: no pruning.
+                                          Scores are cumulative log-probabilities on both sides; with
+                                          DBA_FLAG_PRUNE_NORMALISED a completed hypothesis enters the comparison
+                                          (as the reference and as the one tested) with score / length, as
+                                          Section 4 normalises completed hypotheses before it prunes; the beam
+                                          stays ordered by cumulative score either way                       */
 } dba_config;
 
 /*
@@ -156,6 +164,19 @@ dba_status dba_step(dba_handle* h, const void* logits_dev, int64_t row_stride_el
                     const float* row_lse_in_dev, const dba_step_out* out_dev);
 
 /*
+ * The same step fused into its producer (Section 2: the k x |V_T| matrix is DECODER-STEP's output, the decoder's
+ * final hidden states times the output embedding): the caller passes the hidden states of the R = B*k hypotheses and
+ * the embedding, the logits are computed on the tensor cores and consumed as they appear (see dba_project_scan for
+ * shapes, alignment and accuracy), and the rest of the step is dba_step's.  Needs DBA_FLAG_FUSED_PROJECTION.
+ *   hidden_dev [B*k, D] bf16, row r = hypothesis in beam slot r;  embed_dev [V, D] bf16.
+ * Every row is projected, open or not.  One corner differs from dba_step: when a row's scores are equal over a run
+ * that reaches past the k+2 entries kept of the row, dba_step looks the row up again to find the lowest word ids
+ * of the run; here there is no row to look up, the kept entries stand, and counters[1] of dba_counters counts it.
+ */
+dba_status dba_step_fused(dba_handle* h, const void* hidden_dev, int64_t hidden_stride_elems, const void* embed_dev,
+                          int64_t embed_stride_elems, int32_t D, const dba_step_out* out_dev);
+
+/*
  * The same step with HOST buffers: copies the logits to a staging area in the workspace, runs the
  * step, copies the requested outputs back and synchronises the stream.  Needs DBA_FLAG_HOST_STAGING.
  * Pinned host memory makes the copies asynchronous with respect to the host until the final wait.
@@ -188,15 +209,27 @@ dba_status dba_timing_read(dba_handle* h, double ms_total[3], int64_t* steps);
 
 /*
  * Diagnostic counters of the handle's device status block (never an error).  Synchronises the stream.
- *   counters[0]  row segments whose K1 best entries the row scan had to find by a second, slow pass over global
+ *   counters[0]  row segments whose k+2 best entries the row scan had to find by a second, slow pass over global
  *                memory, because more entries tied at its selection bound than its lists hold (long runs of
  *                equal logits).  Results are exact either way; a large count explains a slow step.
- *   counters[1..3]  reserved, 0.
+ *   counters[1]  dba_step_fused only: rows whose run of equal scores reached past the kept entries (see there).
+ *   counters[2..3]  reserved, 0.
  */
 dba_status dba_counters(dba_handle* h, uint32_t counters[4]);
 
 /* Number of kernels this handle has launched so far (for accounting in benchmarks). */
 uint64_t dba_launch_count(const dba_handle* h);
+
+/*
+ * Testing aid (no step of the method): shortens the bounded device-side waits of the streaming row scan and
+ * can make one of them run out, so that the DBA_ERR_TIMEOUT path can be exercised without any fault.
+ *   wait_clocks  > 0: GPU clocks a wait may last before the kernel gives up (default: about a second)
+ *   drop_item    >= 0: every thread block announces the copy of this item (a stretch of up to 44 KB of a row) of
+ *                its sequence but does not issue it, so the wait for it runs out after wait_clocks; the kernel
+ *                then records the failure and returns (nothing faults or hangs).  < 0: every copy is issued.
+ * h == NULL sets the two for the stand-alone scans of this process (dba_row_scan, dba_row_scan_static).
+ */
+dba_status dba_test_hook(dba_handle* h, int64_t wait_clocks, int32_t drop_item);
 
 /* Frees the handle (not the workspace). NULL is allowed. */
 void dba_destroy(dba_handle* h);
@@ -210,11 +243,35 @@ const char* dba_status_string(dba_status s);
  *   row_lse_dev [R] fp32;  top_val_dev [R, n_top] fp32 (widened);  top_idx_dev [R, n_top] int32.
  * If V < n_top the tail is filled with (-inf, -1).  scratch_dev must hold dba_row_scan_scratch_bytes.
  * Enqueues on `cuda_stream`, does not synchronise.  n_top <= 66.
+ * Failure of a device-side wait (a copy that never arrived; see DBA_ERR_TIMEOUT) cannot be returned by a call
+ * that does not synchronise: in that case EVERY row's result is replaced by row_lse = NaN and a list of
+ * (-inf, -1), which no successful scan produces (a row without finite entries has row_lse = -inf).
  */
 dba_status dba_row_scan_scratch_bytes(int32_t R, int32_t V, int32_t n_top, int32_t logit_dtype, size_t* bytes);
 dba_status dba_row_scan(const void* logits_dev, int32_t logit_dtype, int32_t R, int32_t V,
                         int64_t row_stride_elems, int32_t n_top, void* scratch_dev, size_t scratch_bytes,
                         float* row_lse_dev, float* top_val_dev, int32_t* top_idx_dev, void* cuda_stream);
+
+/*
+ * The row scan fused into the step before it (Section 2: the k x |V_T| matrix is the output of DECODER-STEP, whose
+ * last stage multiplies the decoder's final hidden states by the output embedding).  logits[r, w] =
+ * sum_j hidden[r, j] * embed[w, j] are computed on the tensor cores (bf16 operands, fp32 accumulation) and consumed
+ * as they are produced: the R x V matrix is never written to memory.  Results as for dba_row_scan, for the logits so
+ * defined (they agree with a double-precision evaluation of the inner products to within the rounding of an fp32
+ * accumulation over D terms; where two logits are closer than that, their order in the list may differ from the
+ * exactly evaluated one).
+ *   hidden_dev [R, D] bf16, rows hidden_stride_elems apart;  embed_dev [V, D] bf16, rows embed_stride_elems apart;
+ *   both 16-byte aligned with strides that are multiples of 8 elements; D a multiple of 8.  n_top <= 32.
+ *   Other shapes: DBA_ERR_UNSUPPORTED.  scratch_dev must hold dba_project_scan_scratch_bytes (for the current device).
+ * Enqueues on `cuda_stream`, does not synchronise.  A failed device-side wait, or a row with more than 64 logits tied
+ * at its n_top-th largest value inside one stretch of the vocabulary, is reported as for dba_row_scan: every row's
+ * result is replaced by row_lse = NaN and a list of (-inf, -1).
+ */
+dba_status dba_project_scan_scratch_bytes(int32_t R, int32_t V, int32_t n_top, size_t* bytes);
+dba_status dba_project_scan(const void* hidden_dev, int64_t hidden_stride_elems, const void* embed_dev,
+                            int64_t embed_stride_elems, int32_t R, int32_t V, int32_t D, int32_t n_top,
+                            void* scratch_dev, size_t scratch_bytes, float* row_lse_dev, float* top_val_dev,
+                            int32_t* top_idx_dev, void* cuda_stream);
 
 /*
  * dba_row_scan for callers that cannot allocate device memory (the paper has no counterpart: this is a

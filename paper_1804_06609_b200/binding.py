@@ -12,11 +12,11 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libdba.so")
 
 F32, BF16 = 0, 1
-FLAG_ADJUST_OFF, FLAG_LENGTH_NORM, FLAG_HOST_STAGING = 1, 2, 4
+FLAG_ADJUST_OFF, FLAG_LENGTH_NORM, FLAG_HOST_STAGING, FLAG_PRUNE_NORMALISED, FLAG_FUSED_PROJECTION = 1, 2, 4, 8, 16
 
-EXPORTS = ["dba_workspace_bytes", "dba_init", "dba_reset", "dba_step", "dba_step_host", "dba_finalize",
-           "dba_timing_enable", "dba_timing_read", "dba_counters", "dba_launch_count", "dba_destroy", "dba_status_string", "dba_row_scan_scratch_bytes", "dba_row_scan",
-           "dba_row_scan_static", "dba_row_scan_static_max_bytes"]
+EXPORTS = ["dba_workspace_bytes", "dba_init", "dba_reset", "dba_step", "dba_step_fused", "dba_step_host", "dba_finalize",
+           "dba_timing_enable", "dba_timing_read", "dba_counters", "dba_launch_count", "dba_test_hook", "dba_destroy", "dba_status_string", "dba_row_scan_scratch_bytes", "dba_row_scan",
+           "dba_row_scan_static", "dba_row_scan_static_max_bytes", "dba_project_scan_scratch_bytes", "dba_project_scan"]
 
 
 class DbaError(RuntimeError):
@@ -53,12 +53,14 @@ def lib():
         L.dba_reset.argtypes = [vp]
         L.dba_step.argtypes = [vp, vp, C.c_int64, vp, C.POINTER(StepOut)]
         L.dba_step_host.argtypes = [vp, vp, C.c_int64, C.POINTER(StepOut)]
+        L.dba_step_fused.argtypes = [vp, vp, C.c_int64, vp, C.c_int64, C.c_int32, C.POINTER(StepOut)]
         L.dba_finalize.argtypes = [vp, vp, vp, vp, vp]
         L.dba_timing_enable.argtypes = [vp, C.c_int32]
         L.dba_timing_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.dba_counters.argtypes = [vp, C.POINTER(C.c_uint32)]
         L.dba_launch_count.argtypes = [vp]
         L.dba_launch_count.restype = C.c_uint64
+        L.dba_test_hook.argtypes = [vp, C.c_int64, C.c_int32]
         L.dba_destroy.argtypes = [vp]
         L.dba_destroy.restype = None
         L.dba_status_string.argtypes = [C.c_int]
@@ -68,6 +70,9 @@ def lib():
                                    vp, vp, vp, vp]
         L.dba_row_scan_static.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int32, vp, vp, vp, vp]
         L.dba_row_scan_static_max_bytes.restype = C.c_size_t
+        L.dba_project_scan_scratch_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_size_t)]
+        L.dba_project_scan.argtypes = [vp, C.c_int64, vp, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp, C.c_size_t,
+                                       vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -153,6 +158,19 @@ class DbaStepper:
         _check(lib().dba_step(self._h, logits.data_ptr(), logits.stride(0), lse_ptr, C.byref(so)), "dba_step")
         return out
 
+    def step_fused(self, hidden, embed, out=None):
+        """hidden: CUDA bfloat16 [B*k, D]; embed: CUDA bfloat16 [V, D].  The step on logits = hidden @ embed.T, which are
+        never materialised.  The stepper must have been made with FLAG_FUSED_PROJECTION."""
+        torch = self.torch
+        assert hidden.is_cuda and embed.is_cuda and hidden.dtype == torch.bfloat16 and embed.dtype == torch.bfloat16
+        assert hidden.shape[0] == self.R and embed.shape[0] == self.V and hidden.shape[1] == embed.shape[1]
+        assert hidden.stride(1) == 1 and embed.stride(1) == 1
+        out = self.out if out is None else out
+        so = self._out_struct(out)
+        _check(lib().dba_step_fused(self._h, hidden.data_ptr(), hidden.stride(0), embed.data_ptr(), embed.stride(0),
+                                    hidden.shape[1], C.byref(so)), "dba_step_fused")
+        return out
+
     def step_host(self, logits_host, out_host):
         """logits_host: CPU tensor [B*k, V] (pinned for asynchronous copies); out_host: dict of CPU tensors."""
         assert not logits_host.is_cuda and logits_host.shape == (self.R, self.V) and logits_host.stride(1) == 1
@@ -181,6 +199,10 @@ class DbaStepper:
         out = (C.c_uint32 * 4)()
         _check(lib().dba_counters(self._h, out), "dba_counters")
         return list(out)
+
+    def test_hook(self, wait_clocks=0, drop_item=-1):
+        """Testing aid: shortens the row scan's bounded waits and can make one run out (see dba_test_hook)."""
+        _check(lib().dba_test_hook(self._h, wait_clocks, drop_item), "dba_test_hook")
 
     def launch_count(self):
         return int(lib().dba_launch_count(self._h))
@@ -214,12 +236,41 @@ def row_scan(logits, n_top, stream=None):
     return lse, val, idx
 
 
+def project_scan(hidden, embed, n_top, stream=None):
+    """Fused output projection + row scan: hidden [R, D] and embed [V, D] (CUDA, bfloat16, unit inner stride).  Per
+    row of hidden @ embed.T: log-sum-exp and the n_top largest logits, as row_scan returns them."""
+    import torch
+    assert hidden.is_cuda and embed.is_cuda and hidden.dtype == torch.bfloat16 and embed.dtype == torch.bfloat16
+    assert hidden.dim() == 2 and embed.dim() == 2 and hidden.shape[1] == embed.shape[1]
+    assert hidden.stride(1) == 1 and embed.stride(1) == 1 and hidden.device == embed.device
+    R, D = hidden.shape
+    V = embed.shape[0]
+    with torch.cuda.device(hidden.device):
+        n = C.c_size_t()
+        _check(lib().dba_project_scan_scratch_bytes(R, V, n_top, C.byref(n)), "dba_project_scan_scratch_bytes")
+        scratch = torch.empty(n.value + 256, dtype=torch.uint8, device=hidden.device)
+        base = (scratch.data_ptr() + 255) // 256 * 256
+        lse = torch.empty(R, dtype=torch.float32, device=hidden.device)
+        val = torch.empty(R, n_top, dtype=torch.float32, device=hidden.device)
+        idx = torch.empty(R, n_top, dtype=torch.int32, device=hidden.device)
+        st = stream if stream is not None else torch.cuda.current_stream(hidden.device)
+        _check(lib().dba_project_scan(hidden.data_ptr(), hidden.stride(0), embed.data_ptr(), embed.stride(0), R, V, D, n_top,
+                                      base, n.value, lse.data_ptr(), val.data_ptr(), idx.data_ptr(), st.cuda_stream),
+               "dba_project_scan")
+        st.synchronize()          # the scratch tensor must outlive the kernels
+    return lse, val, idx
+
+
 def row_scan_static(logits, n_top, lse, val, idx, stream=None):
     """dba_row_scan_static: like row_scan, but the library's built-in scratch is used and the caller brings the
     output tensors (lse [R] f32, val [R, n_top] f32, idx [R, n_top] i32).  Nothing is allocated here."""
     import torch
+    assert logits.is_cuda and logits.dim() == 2 and logits.stride(1) == 1
     R, V = logits.shape
-    st = stream if stream is not None else torch.cuda.current_stream(logits.device)
-    _check(lib().dba_row_scan_static(logits.data_ptr(), _dtype_code(logits), R, V, logits.stride(0), n_top,
-                                     lse.data_ptr(), val.data_ptr(), idx.data_ptr(), st.cuda_stream),
-           "dba_row_scan_static")
+    for t, shape, dt in ((lse, (R,), torch.float32), (val, (R, n_top), torch.float32), (idx, (R, n_top), torch.int32)):
+        assert t.is_cuda and t.device == logits.device and t.dtype == dt and tuple(t.shape) == shape and t.is_contiguous()
+    with torch.cuda.device(logits.device):         # the library looks its scratch up on the current device
+        st = stream if stream is not None else torch.cuda.current_stream(logits.device)
+        _check(lib().dba_row_scan_static(logits.data_ptr(), _dtype_code(logits), R, V, logits.stride(0), n_top,
+                                         lse.data_ptr(), val.data_ptr(), idx.data_ptr(), st.cuda_stream),
+               "dba_row_scan_static")

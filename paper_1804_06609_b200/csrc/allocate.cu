@@ -8,9 +8,14 @@ namespace dba {
 namespace {
 
 // Algorithm 1, DECODER-INIT: slot 0 holds the start symbol at score 0, the other slots are empty.
-__global__ void reset_kernel(Dims d, Beam beam, int32_t* __restrict__ open_list, int32_t* __restrict__ open_count) {
+__global__ void reset_kernel(Dims d, Beam beam, int32_t* __restrict__ open_list, int32_t* __restrict__ open_count,
+                             RowTop top) {
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= d.R) return;
+    // the row lists start out empty and well-formed, so that a scan that fails (a wait that ran out) leaves the
+    // candidate kernel nothing it could misread
+    top.lse[r] = 0.f;
+    for (int e = 0; e < d.K1; ++e) { top.val[(int64_t)r * d.K1 + e] = neg_inf(); top.idx[(int64_t)r * d.K1 + e] = -1; }
     const bool first = (r % d.k) == 0;
     beam.score[r] = first ? 0.f : neg_inf();
     beam.token[r] = first ? d.bos_id : d.pad_id;
@@ -66,8 +71,8 @@ __global__ void finalize_kernel(Dims d, Beam beam, const int32_t* __restrict__ h
 }  // namespace
 
 cudaError_t launch_reset(const Dims& d, const Beam& beam, int32_t* open_list, int32_t* open_count,
-                         cudaStream_t st, int* launches) {
-    reset_kernel<<<(d.R + 255) / 256, 256, 0, st>>>(d, beam, open_list, open_count);
+                         const RowTop& top, cudaStream_t st, int* launches) {
+    reset_kernel<<<(d.R + 255) / 256, 256, 0, st>>>(d, beam, open_list, open_count, top);
     ++*launches;
     return cudaGetLastError();
 }

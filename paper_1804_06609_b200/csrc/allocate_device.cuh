@@ -35,7 +35,8 @@ struct AllocIn {
 };
 
 // One warp.  Writes the sentence's new beam (and the requested outputs, the history, the stop bits) and appends
-// its open rows to the list the next step's row scan reads.
+// its open rows to the list the next step's row scan reads (the order of that list varies from run to run; no
+// result depends on it).
 __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, const AllocIn& in, const Beam& nxt,
                                                   const float* __restrict__ row_lse, const dba_step_out& out,
                                                   int32_t* __restrict__ hist_bp, int32_t* __restrict__ hist_tok,
@@ -47,6 +48,7 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
     __shared__ float a_score[kMaxK];
     __shared__ int a_flat[kMaxK];
     __shared__ int a_tok[kMaxK];
+    __shared__ float a_val[kMaxK];     // what a hypothesis enters the pruning comparison with
     const int lane = threadIdx.x & 31;
     const int k = d.k, V = d.V;
     const int* bank_cnt = in.bank_cnt; const int* order = in.order;
@@ -139,27 +141,40 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
     const int ns = off[0];
     for (int i = lane; i < ns; i += 32) { const int id = order[sel[i]]; sel[i] = id; a_score[i] = c_score[id]; a_flat[i] = c_flat[id]; }
     __syncwarp();
-    // Section 4: threshold pruning.  Hypotheses scoring below (best completed score - threshold) are removed,
-    // completed or not; they are the tail of the ordered beam, so their slots are simply left empty.
+    // Section 4: threshold pruning.  Hypotheses whose value is below (best completed value - threshold) are
+    // removed, completed or not, and the ones behind them move up.  The value is the cumulative score; with
+    // DBA_FLAG_PRUNE_NORMALISED a completed hypothesis enters with score / length on both sides of the comparison.
     float cut = neg_inf();
     if (d.prune > 0.f) {
         float best = neg_inf();
         for (int i = lane; i < ns; i += 32) {
             const int fi = a_flat[i];
-            if (fi - (fi / V) * V == d.eos_id) best = fmaxf(best, a_score[i]);
+            const int h = fi / V, w = fi - h * V;
+            float v = a_score[i];
+            if (w == d.eos_id) {
+                if (d.flags & DBA_FLAG_PRUNE_NORMALISED) {
+                    const int len = par_kind[h] == 2 ? par_len[h] : par_len[h] + 1;
+                    if (len > 0) v = __fdiv_rn(v, (float)len);
+                }
+                best = fmaxf(best, v);
+            }
+            a_val[i] = v;
         }
         best = warp_max(best);
         if (best != neg_inf()) cut = __fsub_rn(best, d.prune);
+        __syncwarp();
     }
     // new beam in decreasing score order, ties by lower flat index (Section 3.1), empty slots last
     const int r0 = b * k;
+    const bool pruning = cut != neg_inf();
     int n_pruned = 0;
-    for (int i0 = 0; i0 < ns; i0 += 32) n_pruned += __popc(__ballot_sync(kFullMask, i0 + lane < ns && a_score[i0 + lane] < cut));
+    if (pruning)
+        for (int i0 = 0; i0 < ns; i0 += 32) n_pruned += __popc(__ballot_sync(kFullMask, i0 + lane < ns && a_val[i0 + lane] < cut));
     for (int i = lane; i < k; i += 32) {
-        if (i < ns && !(a_score[i] < cut)) {
+        if (i < ns && !(pruning && a_val[i] < cut)) {
             const float si = a_score[i]; const int fi = a_flat[i];
             int rank = 0;
-            for (int j = 0; j < ns; ++j) rank += cell_better(a_score[j], a_flat[j], si, fi);
+            for (int j = 0; j < ns; ++j) rank += cell_better(a_score[j], a_flat[j], si, fi) && !(pruning && a_val[j] < cut);
             const int id = sel[i];
             const uint64_t cmask = c_mask[id]; const int cactive = c_active[id];
             const int h = fi / V, w = fi - h * V;

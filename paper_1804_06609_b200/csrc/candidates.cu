@@ -85,13 +85,16 @@ __device__ __forceinline__ uint64_t merge_top32(uint64_t a, uint64_t b, int lane
 // 48 registers: two CTAs of 672 threads (a warp per row at k = 20, and one more) fit an SM.
 __global__ void __maxnreg__(48)
 candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const SentCons* __restrict__ cons,
-                  Beam cur, Beam nxt, ScanOut part, const float* __restrict__ lse_in, float* __restrict__ row_lse,
-                  dba_step_out out, int32_t* __restrict__ hist_bp, int32_t* __restrict__ hist_tok,
+                  Beam cur, Beam nxt, RowTop top, ScanScratch part, const float* __restrict__ lse_in,
+                  const float* __restrict__ s2_given, dba_step_out out, int32_t* __restrict__ hist_bp, int32_t* __restrict__ hist_tok,
                   uint32_t* __restrict__ status, int32_t* __restrict__ open_list, int32_t* __restrict__ open_count) {
     extern __shared__ __align__(16) unsigned char smem[];
-    const int k = d.k, V = d.V, K1 = d.K1, S = d.S;
+    const int k = d.k, V = d.V, K1 = d.K1;
+    const int S = part.m ? d.S : 0;     // > 0: the streaming scan left one partial result per (row, segment) in `part`;
+                                        // 0: the row's finished list and normaliser are in `top`
+    float* row_lse = top.lse;      // written by the row scan for open rows; set to 0 here for the others
     const int n_threads = blockDim.x, n_warps = n_threads >> 5;
-    const Layout L = make_layout(k, K1, S, d.max_cand, n_warps);
+    const Layout L = make_layout(k, K1, d.S, d.max_cand, n_warps);
     SentCons& sc = *reinterpret_cast<SentCons*>(smem + L.cons);
     uint64_t* s_mask = reinterpret_cast<uint64_t*>(smem + L.mask);
     float* s_parent = reinterpret_cast<float*>(smem + L.parent);
@@ -162,7 +165,9 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
                             if (!((m >> e) & 1ull)) { ok = false; break; }
                     }
                 }
-                s2_x[h * kMaxC + j] = ok ? load_logit_dyn(logits, d.dtype, (int64_t)(r0 + h) * stride + sc.ctok[j]) : neg_inf();
+                // (with the projection fused into the step there is no logit matrix: the logits of the constraint
+                //  tokens were computed on their own and are read further down, once they are there)
+                s2_x[h * kMaxC + j] = !ok ? neg_inf() : logits ? load_logit_dyn(logits, d.dtype, (int64_t)(r0 + h) * stride + sc.ctok[j]) : 0.f;
             }
         }
     }
@@ -172,10 +177,15 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     __syncthreads();
     const int C = sc.C;
     if (tid < k) s_eos_ok[tid] = __popcll(s_mask[tid]) >= C;   // Section 3.3: end token only once all are met
+    if (!logits)
+        for (int q = tid; q < k * kMaxC; q += n_threads) {
+            const int h = q >> 6, j = q & 63;
+            if (s_kind[h] == 1 && j < C && s2_x[q] != neg_inf()) s2_x[q] = s2_given[(int64_t)(r0 + h) * kMaxC + j];
+        }
     __syncthreads();
 
     // ---- phase A: per row, the k best cells in (score desc, token asc) order ------------------------------
-    uint64_t* stage = reinterpret_cast<uint64_t*>(smem + L.stage) + warp * (S > 1 ? S * K1 : 0);
+    uint64_t* stage = reinterpret_cast<uint64_t*>(smem + L.stage) + warp * (d.S > 1 ? d.S * K1 : 0);
     uint64_t* merged = reinterpret_cast<uint64_t*>(smem + L.merged) + warp * K1;
     float* tmp_score = reinterpret_cast<float*>(smem + L.tmp_score) + warp * K1;
     int* tmp_w = reinterpret_cast<int*>(smem + L.tmp_w) + warp * K1;
@@ -190,72 +200,92 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
             if (lane == 0) { rt_n[h] = 1; rt_score[h * k] = s_parent[h]; rt_w[h * k] = d.eos_id; row_lse[r] = 0.f; s_lse[h] = 0.f; }
             continue;
         }
-        // every global load of this row first (they are independent), so that their latencies overlap
-        const int n_ent = S * K1;
-        const float mg = lane < S ? part.m[r * S + lane] : neg_inf();
-        const float sg = lane < S ? part.s[r * S + lane] : 0.f;
-        const float lse_given = lse_in ? lse_in[r] : 0.f;
-        {   // four loads of each array in flight before the first key is stored (the stores would hold them back)
-            uint64_t* dst = S == 1 ? merged : stage;
-            const int32_t* gi = part.top_idx + (int64_t)r * n_ent;
-            const float* gv = part.top_val + (int64_t)r * n_ent;
-            for (int e0 = lane; e0 < n_ent; e0 += 128) {
-                int ix[4]; float xv[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int e = e0 + 32 * q;
-                    ix[q] = e < n_ent ? __ldg(gi + e) : -1;
-                    xv[q] = e < n_ent ? __ldg(gv + e) : 0.f;
-                }
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int e = e0 + 32 * q;
-                    if (e < n_ent) dst[e] = ix[q] >= 0 ? row_key(xv[q], ix[q]) : 0ull;
-                }
-            }
-        }
-        // row normaliser from the segment partials: lane g holds segment g (S <= 8), fixed reduction order
         float lse;
-        {
-            const float M = warp_max(mg);
-            const float sum = warp_sum(mg != neg_inf() ? sg * expf(mg - M) : 0.f);
-            lse = M == neg_inf() ? neg_inf() : M + logf(sum);
-        }
-        if (lane == 0) row_lse[r] = lse;
-        if (lse_in) lse = lse_given;
-        if (lane == 0) s_lse[h] = lse;
-        const float parent = s_parent[h];
-        const bool eos_ok = s_eos_ok[h] != 0;
-
-        // the row's K1 largest raw logits, merged over segments, as keys in `merged`
-        if (S > 1) {
-            const int n = n_ent;
-            for (int e = lane; e < K1; e += 32) merged[e] = 0ull;
-            __syncwarp();
-            if (K1 <= 32) {
-                uint64_t acc = lane < K1 ? stage[lane] : 0ull;
-                for (int g = 1; g < S; ++g) acc = merge_top32(acc, lane < K1 ? stage[g * K1 + lane] : 0ull, lane);
-                if (lane < K1) merged[lane] = acc;
-            } else
-            // every segment's list is in descending key order (empty entries, key 0, last): the place of an
-            // entry in the merged order is its place in its own list plus, for every other list, the number of
-            // keys above it, found by bisection
-            for (int e = lane; e < n; e += 32) {
-                const uint64_t key = stage[e];
-                if (!key) continue;
-                const int g = e / K1;
-                int rank = e - g * K1;
-                for (int g2 = 0; g2 < S; ++g2) {
-                    if (g2 == g) continue;
-                    const uint64_t* lst = stage + g2 * K1;
-                    int lo2 = 0, hi2 = K1;                      // first position whose key is not above `key`
-                    while (lo2 < hi2) { const int mid = (lo2 + hi2) >> 1; if (lst[mid] > key) lo2 = mid + 1; else hi2 = mid; }
-                    rank += lo2;
+        float parent;
+        bool eos_ok;
+        if (S > 0) {
+            // every global load of this row first (they are independent), so that their latencies overlap
+            const int n_ent = S * K1;
+            const float mg = lane < S ? part.m[r * S + lane] : neg_inf();
+            const float sg = lane < S ? part.s[r * S + lane] : 0.f;
+            const float lse_given = lse_in ? lse_in[r] : 0.f;
+            {   // four loads of each array in flight before the first key is stored (the stores would hold them back)
+                uint64_t* dst = S == 1 ? merged : stage;
+                const int32_t* gi = part.idx + (int64_t)r * n_ent;
+                const float* gv = part.val + (int64_t)r * n_ent;
+                for (int e0 = lane; e0 < n_ent; e0 += 128) {
+                    int ix[4]; float xv[4];
+    #pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int e = e0 + 32 * q;
+                        ix[q] = e < n_ent ? __ldg(gi + e) : -1;
+                        xv[q] = e < n_ent ? __ldg(gv + e) : 0.f;
+                    }
+    #pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int e = e0 + 32 * q;
+                        if (e < n_ent) dst[e] = ix[q] >= 0 ? row_key(xv[q], ix[q]) : 0ull;
+                    }
                 }
-                if (rank < K1) merged[rank] = key;
             }
+            // row normaliser from the segment partials: lane g holds segment g (S <= 8), fixed reduction order
+            {
+                const float M = warp_max(mg);
+                const float sum = warp_sum(mg != neg_inf() ? sg * expf(mg - M) : 0.f);
+                lse = M == neg_inf() ? neg_inf() : M + logf(sum);
+            }
+            if (lane == 0) row_lse[r] = lse;
+            if (lse_in) lse = lse_given;
+            if (lane == 0) s_lse[h] = lse;
+            parent = s_parent[h];
+            eos_ok = s_eos_ok[h] != 0;
+
+            // the row's K1 largest raw logits, merged over segments, as keys in `merged`
+            if (S > 1) {
+                const int n = n_ent;
+                for (int e = lane; e < K1; e += 32) merged[e] = 0ull;
+                __syncwarp();
+                if (K1 <= 32) {
+                    uint64_t acc = lane < K1 ? stage[lane] : 0ull;
+                    for (int g = 1; g < S; ++g) acc = merge_top32(acc, lane < K1 ? stage[g * K1 + lane] : 0ull, lane);
+                    if (lane < K1) merged[lane] = acc;
+                } else
+                // every segment's list is in descending key order (empty entries, key 0, last): the place of an
+                // entry in the merged order is its place in its own list plus, for every other list, the number of
+                // keys above it, found by bisection
+                for (int e = lane; e < n; e += 32) {
+                    const uint64_t key = stage[e];
+                    if (!key) continue;
+                    const int g = e / K1;
+                    int rank = e - g * K1;
+                    for (int g2 = 0; g2 < S; ++g2) {
+                        if (g2 == g) continue;
+                        const uint64_t* lst = stage + g2 * K1;
+                        int lo2 = 0, hi2 = K1;                      // first position whose key is not above `key`
+                        while (lo2 < hi2) { const int mid = (lo2 + hi2) >> 1; if (lst[mid] > key) lo2 = mid + 1; else hi2 = mid; }
+                        rank += lo2;
+                    }
+                    if (rank < K1) merged[rank] = key;
+                }
+            }
+            __syncwarp();
+        } else {
+            // the row's K1 largest raw logits (the finished list) as keys in `merged`, and its normaliser
+            lse = row_lse[r];
+            const float lse_given = lse_in ? lse_in[r] : 0.f;
+            const int32_t* gi = top.idx + (int64_t)r * K1;
+            const float* gv = top.val + (int64_t)r * K1;
+            for (int e = lane; e < K1; e += 32) {
+                const int ix = gi[e];
+                const float xv = gv[e];
+                merged[e] = ix >= 0 ? row_key(xv, ix) : 0ull;
+            }
+            if (lse_in) lse = lse_given;
+            if (lane == 0) s_lse[h] = lse;
+            parent = s_parent[h];
+            eos_ok = s_eos_ok[h] != 0;
+            __syncwarp();
         }
-        __syncwarp();
 
         // scores of the entries that may be generated, in list order
         int total_valid = 0, finite_entries = 0;
@@ -301,6 +331,10 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
                 if ((bits << 1) == 0) bits = 0x80000000u | ulp;
                 else bits = (bits & 0x80000000u) ? bits + ulp : bits - ulp;
                 rescan = !(tmp_x[g] == xl && cell_score(__uint_as_float(bits), lse, parent) < sb);
+            }
+            if (rescan && !logits) {       // no logit matrix to look into: the listed entries stand (counted, see dba_counters)
+                if (lane == 0) atomicAdd(status + kStatusWordUnresolved, 1u);
+                rescan = false;
             }
             if (rescan) {      // whole row: the cells scoring exactly sb, lowest token ids first
                 const int need = k - g;
@@ -562,49 +596,44 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
 }  // namespace
 
 // Threads per CTA: 1024 when every sentence gets an SM of its own (then only the latency of one CTA counts);
-// otherwise two CTAs share an SM: 672 threads when the beam has more than 15 rows (a warp per row up to k = 20
+// otherwise two CTAs share an SM: 640 threads when the beam has more than 15 rows (a warp per row up to k = 19
 // beside the warp that runs the tournament), else 512; fewer if the per-warp scratch would not fit shared memory.
-static size_t g_smem_limit = 48 * 1024;     // raised by configure_candidates
-static int g_sm_count = 1;
-static int pick_threads(const Dims& d, size_t smem_limit) {
-    const int first = d.B <= g_sm_count ? kCandMaxThreads : (d.k > 15 ? 640 : 512);
+static int pick_threads(const Dims& d, size_t smem_limit, int sm_count) {
+    const int first = d.B <= sm_count ? kCandMaxThreads : (d.k > 15 ? 640 : 512);
     for (int t = first; t > 256; t = t == 640 ? 512 : t >> 1)
         if ((size_t)make_layout(d.k, d.K1, d.S, d.max_cand, t / 32).total <= smem_limit) return t;
     return 256;
 }
 
-size_t candidates_smem_bytes(const Dims& d) { return (size_t)make_layout(d.k, d.K1, d.S, d.max_cand, 256 / 32).total; }
-
 // The dynamic shared memory a block may ask for is the device's opt-in limit less what the kernel declares
 // statically.  *fits = false (and nothing configured) when even the smallest block is over it.
-cudaError_t configure_candidates(const Dims& d, bool* fits) {
-    int dev = 0, lim = 0;
+cudaError_t configure_candidates(const Dims& d, CandLaunch* cl, bool* fits) {
+    int dev = 0, lim = 0, sms = 1;
     *fits = false;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&lim, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaFuncAttributes fa{};
     if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, candidates_kernel);
     if (e != cudaSuccess) return e;
-    g_smem_limit = (size_t)lim > fa.sharedSizeBytes ? (size_t)lim - fa.sharedSizeBytes : 0;
-    e = cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-    if (candidates_smem_bytes(d) > g_smem_limit) return cudaSuccess;
+    const size_t smem_limit = (size_t)lim > fa.sharedSizeBytes ? (size_t)lim - fa.sharedSizeBytes : 0;
+    if ((size_t)make_layout(d.k, d.K1, d.S, d.max_cand, 256 / 32).total > smem_limit) return cudaSuccess;
     *fits = true;
+    cl->threads = pick_threads(d, smem_limit, sms);
+    cl->smem = (size_t)make_layout(d.k, d.K1, d.S, d.max_cand, cl->threads / 32).total;
     // The attribute belongs to the kernel, not to a handle: it is raised to the most any shape may ask for, so
     // that handles of different shapes can be alive together.
-    return cudaFuncSetAttribute(candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g_smem_limit);
+    return cudaFuncSetAttribute(candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_limit);
 }
 
 cudaError_t launch_candidates(const void* logits, int64_t stride, const Dims& d, const SentCons* cons,
-                              const Beam& cur, const Beam& next, const ScanOut& part, const float* lse_in,
-                              float* row_lse, const dba_step_out& out, int32_t* hist_bp, int32_t* hist_tok,
-                              uint32_t* status, int32_t* open_list, int32_t* open_count, cudaStream_t st,
+                              const Beam& cur, const Beam& next, const RowTop& top, const ScanScratch& part,
+                              const float* lse_in, const float* s2_given, const dba_step_out& out, int32_t* hist_bp, int32_t* hist_tok, uint32_t* status,
+                              int32_t* open_list, int32_t* open_count, const CandLaunch& cl, cudaStream_t st,
                               int* launches) {
-    const int threads = pick_threads(d, g_smem_limit);
-    const size_t smem = (size_t)make_layout(d.k, d.K1, d.S, d.max_cand, threads / 32).total;
     ++*launches;
-    return launch_after(candidates_kernel, dim3(d.B), dim3(threads), smem, st, logits, stride, d, cons, cur, next, part,
-                        lse_in, row_lse, out, hist_bp, hist_tok, status, open_list, open_count);
+    return launch_after(candidates_kernel, dim3(d.B), dim3(cl.threads), cl.smem, st, logits, stride, d, cons, cur, next,
+                        top, part, lse_in, s2_given, out, hist_bp, hist_tok, status, open_list, open_count);
 }
 
 }  // namespace dba

@@ -19,8 +19,13 @@ struct dba_handle {
     Beam beam[2];
     int32_t* hist_bp;
     int32_t* hist_tok;
-    ScanOut part;
-    float* row_lse;
+    RowTop top;                    // the row scan's results (top.lse doubles as the step's row_lse output)
+    ScanScratch part;
+    ProjPieces proj;               // only with DBA_FLAG_FUSED_PROJECTION: scratch of the fused projection
+    int proj_stride;
+    float* s2_logit;               // and the logits of the constraint tokens, [R, 64]
+    CandLaunch cand;               // block size and shared memory of the candidate kernel on this handle's device
+    ScanDebug dbg;
     uint32_t* status;
     int32_t* open_list;            // rows the next step scans, and how many
     int32_t* open_count;           // two counts: step t reads [t & 1], its last kernel fills [(t + 1) & 1]
@@ -39,6 +44,9 @@ struct dba_handle {
 };
 
 constexpr int kTimingCap = 4096;
+
+// testing aids of the stand-alone row scan (dba_test_hook with a null handle)
+static ScanDebug g_scan_debug;
 
 namespace {
 
@@ -64,7 +72,9 @@ dba_status check_config(const dba_config* c, Shape* shape, std::vector<SentCons>
     if (c->B < 1 || c->k < 1 || c->V < 1 || c->max_steps < 1) return DBA_ERR_INVALID_ARG;
     if (c->logit_dtype != DBA_F32 && c->logit_dtype != DBA_BF16) return DBA_ERR_INVALID_ARG;
     if (c->prune_threshold != c->prune_threshold) return DBA_ERR_INVALID_ARG;      // NaN
-    if (c->flags & ~(DBA_FLAG_ADJUST_OFF | DBA_FLAG_LENGTH_NORM | DBA_FLAG_HOST_STAGING)) return DBA_ERR_INVALID_ARG;
+    if (c->flags & ~(DBA_FLAG_ADJUST_OFF | DBA_FLAG_LENGTH_NORM | DBA_FLAG_HOST_STAGING | DBA_FLAG_PRUNE_NORMALISED |
+                     DBA_FLAG_FUSED_PROJECTION))
+        return DBA_ERR_INVALID_ARG;
     const int32_t sp[3] = {c->pad_id, c->bos_id, c->eos_id};
     for (int i = 0; i < 3; ++i)
         if (sp[i] < 0 || sp[i] >= c->V) return DBA_ERR_INVALID_ARG;
@@ -127,21 +137,39 @@ Beam carve_beam(Carver& cv, int R) {
     return b;
 }
 
-// Lays the handle's arrays out in the workspace; sizes use the upper bound max_segments for the segment count.
+RowTop carve_top(Carver& cv, size_t R, int K1) {
+    RowTop t;
+    t.lse = cv.take<float>(R); t.val = cv.take<float>(R * K1); t.idx = cv.take<int32_t>(R * K1);
+    return t;
+}
+
+ScanScratch carve_scratch(Carver& cv, size_t R, int S, int K1) {
+    ScanScratch s;
+    s.m = cv.take<float>(R * S); s.s = cv.take<float>(R * S);
+    s.val = cv.take<float>(R * S * K1); s.idx = cv.take<int32_t>(R * S * K1);
+    return s;
+}
+
+ProjPieces carve_pieces(Carver& cv, size_t R, int P) {
+    ProjPieces q;
+    const size_t cap = (size_t)project_list_cap();
+    q.ref = cv.take<int32_t>(R * P); q.sum = cv.take<float>(R * P); q.n = cv.take<int32_t>(R * P);
+    q.val = cv.take<float>(R * P * cap); q.col = cv.take<int32_t>(R * P * cap);
+    return q;
+}
+
+// Lays the handle's arrays out in the workspace.
 size_t carve(dba_handle* h, void* base, int32_t max_steps) {
     Carver cv(base);
     const Dims& d = h->d;
-    const size_t R = d.R, items = (size_t)d.R * max_segments(d.V, d.dtype);
+    const size_t R = d.R;
     h->cons = cv.take<SentCons>(d.B);
     h->beam[0] = carve_beam(cv, d.R);
     h->beam[1] = carve_beam(cv, d.R);
     h->hist_bp = cv.take<int32_t>(R * max_steps);
     h->hist_tok = cv.take<int32_t>(R * max_steps);
-    h->part.m = cv.take<float>(items);
-    h->part.s = cv.take<float>(items);
-    h->part.top_val = cv.take<float>(items * d.K1);
-    h->part.top_idx = cv.take<int32_t>(items * d.K1);
-    h->row_lse = cv.take<float>(R);
+    h->top = carve_top(cv, R, d.K1);
+    h->part = carve_scratch(cv, R, max_segments(d.V, d.dtype), d.K1);
     h->status = cv.take<uint32_t>(64);
     h->open_list = cv.take<int32_t>(R);
     h->open_count = cv.take<int32_t>(64);
@@ -149,6 +177,13 @@ size_t carve(dba_handle* h, void* base, int32_t max_steps) {
     h->fin_len = cv.take<int32_t>(d.B);
     h->fin_score = cv.take<float>(d.B);
     h->fin_flags = cv.take<int32_t>(d.B);
+    h->s2_logit = nullptr; h->proj_stride = 0;
+    std::memset(&h->proj, 0, sizeof h->proj);
+    if (d.flags & DBA_FLAG_FUSED_PROJECTION) {
+        h->proj_stride = project_pieces(d.R, d.V, h->sm_count);
+        h->proj = carve_pieces(cv, R, h->proj_stride);
+        h->s2_logit = cv.take<float>(R * kMaxC);
+    }
     h->stage_logits = nullptr;
     std::memset(&h->stage_out, 0, sizeof h->stage_out);
     if (d.flags & DBA_FLAG_HOST_STAGING) {
@@ -175,6 +210,12 @@ dba_status dba_workspace_bytes(const dba_config* cfg, size_t* bytes) {
     if (st != DBA_OK) return st;
     dba_handle tmp{};
     fill_dims(cfg, sh, &tmp.d);
+    int dev = 0;
+    tmp.sm_count = 1;
+    if (cfg->flags & DBA_FLAG_FUSED_PROJECTION)      // the projection's scratch depends on the current device's SM count
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&tmp.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return DBA_ERR_CUDA;
     *bytes = carve(&tmp, nullptr, cfg->max_steps);
     return DBA_OK;
 }
@@ -192,22 +233,25 @@ dba_status dba_init(const dba_config* cfg, void* workspace_dev, size_t workspace
     if (!h) return DBA_ERR_INVALID_ARG;
     fill_dims(cfg, sh, &h->d);
     h->max_steps = cfg->max_steps;
-    const size_t need = carve(h, workspace_dev, cfg->max_steps);
-    if (workspace_bytes < need) { delete h; return DBA_ERR_WORKSPACE; }
-    h->stream = (cudaStream_t)cuda_stream;
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
     if (e != cudaSuccess) { delete h; return DBA_ERR_CUDA; }
+    if ((cfg->flags & DBA_FLAG_FUSED_PROJECTION) && h->d.K1 > 32) { delete h; return DBA_ERR_UNSUPPORTED; }
+    const size_t need = carve(h, workspace_dev, cfg->max_steps);
+    if (workspace_bytes < need) { delete h; return DBA_ERR_WORKSPACE; }
+    h->stream = (cudaStream_t)cuda_stream;
     plan_segments(h->d, h->sm_count);
     bool fits = false;
-    e = configure_candidates(h->d, &fits);
+    e = configure_candidates(h->d, &h->cand, &fits);
     if (e == cudaSuccess && !fits) { delete h; return DBA_ERR_UNSUPPORTED; }
     if (e == cudaSuccess) e = configure_row_scan_tma();
+    if (e == cudaSuccess && (cfg->flags & DBA_FLAG_FUSED_PROJECTION)) e = configure_project_scan();
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(h->cons, cons.data(), sizeof(SentCons) * cons.size(), cudaMemcpyHostToDevice, h->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(h->status, 0, 256, h->stream);
     h->launches_tmp = 0;
-    if (e == cudaSuccess) e = launch_reset(h->d, h->beam[0], h->open_list, h->open_count, h->stream, &h->launches_tmp);
+    if (e == cudaSuccess)
+        e = launch_reset(h->d, h->beam[0], h->open_list, h->open_count, h->top, h->stream, &h->launches_tmp);
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);   // `cons` is a local buffer
     if (e != cudaSuccess) { delete h; return DBA_ERR_CUDA; }
     h->launches = h->launches_tmp;
@@ -219,7 +263,8 @@ dba_status dba_init(const dba_config* cfg, void* workspace_dev, size_t workspace
 dba_status dba_reset(dba_handle* h) {
     if (!h) return DBA_ERR_INVALID_ARG;
     h->launches_tmp = 0;
-    cudaError_t e = launch_reset(h->d, h->beam[0], h->open_list, h->open_count, h->stream, &h->launches_tmp);
+    cudaError_t e = launch_reset(h->d, h->beam[0], h->open_list, h->open_count, h->top, h->stream,
+                                 &h->launches_tmp);
     h->launches += h->launches_tmp;
     h->t = 0; h->cur = 0;
     return cuda_fail(e);
@@ -247,17 +292,50 @@ dba_status dba_step(dba_handle* h, const void* logits_dev, int64_t row_stride_el
         h->ev_steps += 1;
     }
     cudaError_t e = cudaSuccess;
+    bool partial = false;
     if (ev) e = cudaEventRecord(ev[0], h->stream);
     if (e == cudaSuccess)
         e = launch_row_scan(logits_dev, row_stride_elems, h->d, cur.score, cur.token, h->open_list,
-                            h->open_count + (h->t & 1), h->open_count + ((h->t + 1) & 1), h->part, h->status,
-                            h->sm_count, h->stream, &h->launches_tmp);
+                            h->open_count + (h->t & 1), h->open_count + ((h->t + 1) & 1), h->top, h->part, h->status,
+                            h->sm_count, h->dbg, h->stream, &h->launches_tmp, &partial);
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[1], h->stream);
+    ScanScratch part = h->part;
+    if (!partial) part.m = nullptr;           // the plain kernel wrote the rows' finished results
     if (e == cudaSuccess)
-        e = launch_candidates(logits_dev, row_stride_elems, h->d, h->cons, cur, nxt, h->part, row_lse_in_dev,
-                              h->row_lse, out, h->hist_bp + (size_t)h->t * h->d.R, h->hist_tok + (size_t)h->t * h->d.R,
-                              h->status, h->open_list, h->open_count + ((h->t + 1) & 1), h->stream, &h->launches_tmp);
+        e = launch_candidates(logits_dev, row_stride_elems, h->d, h->cons, cur, nxt, h->top, part, row_lse_in_dev, nullptr, out,
+                              h->hist_bp + (size_t)h->t * h->d.R, h->hist_tok + (size_t)h->t * h->d.R, h->status,
+                              h->open_list, h->open_count + ((h->t + 1) & 1), h->cand, h->stream, &h->launches_tmp);
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[2], h->stream);
+    h->launches += h->launches_tmp;
+    if (e != cudaSuccess) return DBA_ERR_CUDA;
+    h->cur ^= 1;
+    h->t += 1;
+    return DBA_OK;
+}
+
+dba_status dba_step_fused(dba_handle* h, const void* hidden_dev, int64_t hidden_stride_elems, const void* embed_dev,
+                          int64_t embed_stride_elems, int32_t D, const dba_step_out* out_dev) {
+    if (!h || !hidden_dev || !embed_dev || D < 1 || hidden_stride_elems < D || embed_stride_elems < D) return DBA_ERR_INVALID_ARG;
+    if (!h->s2_logit) return DBA_ERR_STATE;
+    if (h->t >= h->max_steps) return DBA_ERR_STATE;
+    if (!project_scan_usable(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, D, h->d.K1)) return DBA_ERR_UNSUPPORTED;
+    dba_step_out out{};
+    if (out_dev) out = *out_dev;
+    const Beam& cur = h->beam[h->cur];
+    const Beam& nxt = h->beam[h->cur ^ 1];
+    h->launches_tmp = 0;
+    // the list of open rows is not used by this path (every row is projected), but its count is kept in step
+    cudaError_t e = cudaMemsetAsync(h->open_count + ((h->t + 1) & 1), 0, sizeof(int32_t), h->stream);
+    if (e == cudaSuccess)
+        e = launch_project_scan(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, h->d.R, h->d.V, D, h->d.K1,
+                                h->proj, h->proj_stride, h->top, h->status, h->sm_count, h->stream, &h->launches_tmp);
+    if (e == cudaSuccess)
+        e = launch_constraint_logits(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, D, h->d, h->cons,
+                                     h->s2_logit, h->stream, &h->launches_tmp);
+    if (e == cudaSuccess)
+        e = launch_candidates(nullptr, 0, h->d, h->cons, cur, nxt, h->top, ScanScratch{}, nullptr, h->s2_logit, out,
+                              h->hist_bp + (size_t)h->t * h->d.R, h->hist_tok + (size_t)h->t * h->d.R, h->status,
+                              h->open_list, h->open_count + ((h->t + 1) & 1), h->cand, h->stream, &h->launches_tmp);
     h->launches += h->launches_tmp;
     if (e != cudaSuccess) return DBA_ERR_CUDA;
     h->cur ^= 1;
@@ -348,11 +426,18 @@ dba_status dba_counters(dba_handle* h, uint32_t counters[4]) {
     cudaError_t e = cudaMemcpyAsync(words, h->status, sizeof words, cudaMemcpyDeviceToHost, h->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
     if (e != cudaSuccess) return DBA_ERR_CUDA;
-    counters[0] = words[kStatusWordRescans]; counters[1] = counters[2] = counters[3] = 0;
+    counters[0] = words[kStatusWordRescans]; counters[1] = words[kStatusWordUnresolved]; counters[2] = counters[3] = 0;
     return DBA_OK;
 }
 
 uint64_t dba_launch_count(const dba_handle* h) { return h ? h->launches : 0; }
+
+dba_status dba_test_hook(dba_handle* h, int64_t wait_clocks, int32_t drop_item) {
+    ScanDebug& dbg = h ? h->dbg : g_scan_debug;
+    dbg.wait_clocks = wait_clocks > 0 ? (long long)wait_clocks : 0;
+    dbg.drop_item = drop_item >= 0 ? drop_item : -1;
+    return DBA_OK;
+}
 
 void dba_destroy(dba_handle* h) {
     if (!h) return;
@@ -378,8 +463,7 @@ dba_status dba_row_scan_scratch_bytes(int32_t R, int32_t V, int32_t n_top, int32
     if (logit_dtype != DBA_F32 && logit_dtype != DBA_BF16) return DBA_ERR_INVALID_ARG;
     if (n_top > kMaxTop) return DBA_ERR_UNSUPPORTED;
     Carver cv(nullptr);
-    const size_t items = (size_t)R * max_segments(V, logit_dtype);
-    cv.take<float>(items); cv.take<float>(items); cv.take<float>(items * n_top); cv.take<int32_t>(items * n_top);
+    carve_scratch(cv, (size_t)R, max_segments(V, logit_dtype), n_top);
     cv.take<uint32_t>(64);
     *bytes = (cv.off + 255) / 256 * 256;
     return DBA_OK;
@@ -402,19 +486,68 @@ dba_status dba_row_scan(const void* logits_dev, int32_t logit_dtype, int32_t R, 
     plan_segments(d, sms);
     d.K1 = n_top;
     Carver cv(scratch_dev);
-    const size_t items = (size_t)R * max_segments(V, logit_dtype);
-    ScanOut part;
-    part.m = cv.take<float>(items); part.s = cv.take<float>(items);
-    part.top_val = cv.take<float>(items * n_top); part.top_idx = cv.take<int32_t>(items * n_top);
+    ScanScratch part = carve_scratch(cv, (size_t)R, max_segments(V, logit_dtype), n_top);
     uint32_t* status = cv.take<uint32_t>(64);
+    RowTop top;
+    top.lse = row_lse_dev; top.val = top_val_dev; top.idx = top_idx_dev;
     int launches = 0;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // the scratch may hold anything (it may be shared with earlier calls): the status word starts at zero, everything
+    // else is written before it is read
+    bool partial = false;
     e = cudaMemsetAsync(status, 0, 256, stream);
     if (e == cudaSuccess) e = configure_row_scan_tma();
     if (e == cudaSuccess)
-        e = launch_row_scan(logits_dev, row_stride_elems, d, nullptr, nullptr, nullptr, nullptr, nullptr, part, status, sms,
-                            stream, &launches);
-    if (e == cudaSuccess) e = launch_row_merge(d, part, n_top, row_lse_dev, top_val_dev, top_idx_dev, stream, &launches);
+        e = launch_row_scan(logits_dev, row_stride_elems, d, nullptr, nullptr, nullptr, nullptr, nullptr, top, part, status,
+                            sms, g_scan_debug, stream, &launches, &partial);
+    if (e == cudaSuccess && partial) e = launch_row_merge(d, part, n_top, row_lse_dev, top_val_dev, top_idx_dev, stream, &launches);
+    if (e == cudaSuccess) e = launch_scan_check(status, R, n_top, top, stream);
+    return cuda_fail(e);
+}
+
+dba_status dba_project_scan_scratch_bytes(int32_t R, int32_t V, int32_t n_top, size_t* bytes) {
+    if (!bytes || R < 1 || V < 1 || n_top < 1) return DBA_ERR_INVALID_ARG;
+    if (n_top > 32) return DBA_ERR_UNSUPPORTED;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return DBA_ERR_CUDA;
+    Carver cv(nullptr);
+    carve_pieces(cv, (size_t)R, project_pieces(R, V, sms));
+    cv.take<uint32_t>(64);
+    *bytes = (cv.off + 255) / 256 * 256;
+    return DBA_OK;
+}
+
+dba_status dba_project_scan(const void* hidden_dev, int64_t hidden_stride_elems, const void* embed_dev,
+                            int64_t embed_stride_elems, int32_t R, int32_t V, int32_t D, int32_t n_top,
+                            void* scratch_dev, size_t scratch_bytes, float* row_lse_dev, float* top_val_dev,
+                            int32_t* top_idx_dev, void* cuda_stream) {
+    size_t need = 0;
+    dba_status st = dba_project_scan_scratch_bytes(R, V, n_top, &need);
+    if (st != DBA_OK) return st;
+    if (!hidden_dev || !embed_dev || !row_lse_dev || !top_val_dev || !top_idx_dev || D < 1 || hidden_stride_elems < D ||
+        embed_stride_elems < D)
+        return DBA_ERR_INVALID_ARG;
+    if (!project_scan_usable(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, D, n_top)) return DBA_ERR_UNSUPPORTED;
+    if (!scratch_dev || ((uintptr_t)scratch_dev & 255u) || scratch_bytes < need) return DBA_ERR_WORKSPACE;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return DBA_ERR_CUDA;
+    Carver cv(scratch_dev);
+    const int stride = project_pieces(R, V, sms);
+    ProjPieces pieces = carve_pieces(cv, (size_t)R, stride);
+    uint32_t* status = cv.take<uint32_t>(64);
+    RowTop top;
+    top.lse = row_lse_dev; top.val = top_val_dev; top.idx = top_idx_dev;
+    int launches = 0;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    e = cudaMemsetAsync(status, 0, 256, stream);
+    if (e == cudaSuccess) e = configure_project_scan();
+    if (e == cudaSuccess)
+        e = launch_project_scan(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, R, V, D, n_top, pieces, stride,
+                                top, status, sms, stream, &launches);
+    if (e == cudaSuccess) e = launch_scan_check(status, R, n_top, top, stream);
     return cuda_fail(e);
 }
 

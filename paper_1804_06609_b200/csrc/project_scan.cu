@@ -1,0 +1,509 @@
+// Output projection fused with the row scan (Section 2: DECODER-STEP's last stage produces the k x |V_T| matrix
+// that Algorithm 2 reads): logits[r, w] = <hidden[r, :], embed[w, :]> are computed on the tensor cores and
+// consumed where they appear, so the R x V matrix never exists in HBM.
+//
+// One persistent CTA per SM.  The tiles (128 rows of hidden states x 256 words) are numbered row block by row
+// block and dealt out in equal contiguous runs, so a CTA works through part of one row block's vocabulary (and
+// possibly the start of the next row block's).  Roles, talking through mbarriers only:
+//   warp 0    one thread issues the TMA loads (cp.async.bulk.tensor, no multicast) of the 64-deep slices of both
+//             operands into a ring of shared-memory stages (128-byte swizzle);
+//   warp 1    allocates tensor memory; one thread issues tcgen05.mma (128 x 256 x 16, bf16 in, fp32 out) into one
+//             of two accumulators in tensor memory and commits the stage back to the loader;
+//   warps 4-7 the epilogue: thread t owns row t of the tile.  It reads its 256 logits from tensor memory, 32 at a
+//             time, and keeps, over all the tiles of its run: the sum of 2^(x log2e - c) against a whole-number
+//             reference c (raised with an exact rescaling when a logit exceeds it), and the candidates for the row's
+//             K1 largest logits.  Selection: logits at or above a bound tau (-inf at first) go to the thread's list
+//             in shared memory; when some list of the warp has fewer than 32 places left, every thread of the warp
+//             raises its tau to the K1-th largest entry of its list (to 16 bits, by a radix selection over the
+//             list) and drops what fell below, so a list settles at K1 entries plus whatever arrived since.
+// At the end of its part of a row block the thread writes its sum and its list (at least K1 entries, all that reach
+// the final tau) as one piece of the row; project_merge_kernel orders the pieces of a row exactly and writes
+// the row's normaliser and its K1 best entries in the row scan's format.
+// Every wait on an mbarrier is bounded: a wait that runs out sets the timeout bit of the status word and the
+// CTA winds down (the tensor memory is freed on every path).
+#include <climits>
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "dba_device.cuh"
+#include "dba_internal.h"
+
+namespace dba {
+
+namespace {
+
+constexpr int kBM = 128;                 // rows of hidden states per tile (= lanes of tensor memory)
+constexpr int kBN = 256;                 // words per tile (= columns of one accumulator)
+constexpr int kBK = 64;                  // depth of a stage: 64 bf16 = 128 bytes, one swizzle row
+constexpr int kPStages = 3;
+constexpr int kStageA = kBM * kBK * 2;   // 16 KB
+constexpr int kStageB = kBN * kBK * 2;   // 32 KB
+constexpr int kListCap = 64;             // candidates a thread may hold
+constexpr int kEpiThreads = 128;
+constexpr int kProjThreads = 256;
+constexpr int kTmemCols = 512;           // two accumulators of 256 columns
+constexpr long long kProjWaitClocks = 4000000000LL;      // about two seconds: a wait this long has failed
+
+struct ProjSmem {
+    alignas(1024) unsigned char a[kPStages][kStageA];
+    alignas(1024) unsigned char b[kPStages][kStageB];
+    uint32_t list_key[kListCap][kEpiThreads];   // entry e of thread t at [e][t] (no bank conflicts): the logit as an ordered integer
+    int32_t list_col[kListCap][kEpiThreads];
+    uint64_t full[kPStages];         // the stage's operands have landed
+    uint64_t empty[kPStages];        // the stage's MMAs are done
+    uint64_t acc_full[2];            // the accumulator holds a finished tile
+    uint64_t acc_empty[2];           // the epilogue has read the accumulator
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+struct ProjParams {
+    int R, V, D, K1;
+    int tiles_m, tiles_n;            // tiles along rows and along the vocabulary
+    int pieces;                      // most pieces a row may have (stride of the per-piece arrays)
+    ProjPieces out;
+    uint32_t* status;
+};
+
+__device__ __forceinline__ uint32_t psmem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void pbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void pbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void pbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool pbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  False: the CTA is winding down (this wait ran out, or another one did).
+__device__ __noinline__ bool pbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (pbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kProjWaitClocks) break;
+    }
+    *abort_flag = 1;
+    return false;
+}
+// 2-D tiled TMA load (no multicast): box at (x = element along the row, y = row) of the tensor map
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// Shared-memory operand descriptor of a K-major tile stored as rows of 128 bytes with the 128-byte swizzle:
+// start address, leading offset 1 (unused with a swizzle), 1024 bytes from one group of eight rows to the next,
+// descriptor version 1, layout type "128-byte swizzle".
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 128, dense, no negation.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(kIdesc), "r"(accumulate) : "memory");
+}
+// arrives on the mbarrier once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// 32 consecutive columns of this thread's lane of tensor memory
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* r) {
+    uint32_t u[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+          "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
+          "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
+          "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
+}
+__device__ __forceinline__ float pex2(float t) { float r; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t)); return r; }
+__device__ __forceinline__ float ppow2i(int d) { return d < -126 ? 0.f : __int_as_float((d + 127) << 23); }
+
+constexpr float kPLog2e = 1.44269502162933349609375f;
+constexpr float kPNoRef = -1.0e30f;
+
+__global__ void __launch_bounds__(kProjThreads, 1)
+project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, ProjParams p) {
+    extern __shared__ __align__(1024) unsigned char psmem_raw[];
+    // the operand tiles want 1024-byte alignment (the swizzle pattern repeats every 1024 bytes)
+    ProjSmem& sm = *reinterpret_cast<ProjSmem*>(psmem_raw + ((1024u - (psmem_u32(psmem_raw) & 1023u)) & 1023u));
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    volatile int* abort_flag = &sm.abort_flag;
+
+    // this CTA's run of tiles
+    const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
+    const int t_begin = (int)((long long)blockIdx.x * n_tiles / gridDim.x);
+    const int t_end = (int)((long long)(blockIdx.x + 1) * n_tiles / gridDim.x);
+    const int k_blocks = (p.D + kBK - 1) / kBK;
+
+    if (tid == 0) {
+        for (int s = 0; s < kPStages; ++s) { pbar_init(psmem_u32(&sm.full[s]), 1); pbar_init(psmem_u32(&sm.empty[s]), 1); }
+        for (int a = 0; a < 2; ++a) { pbar_init(psmem_u32(&sm.acc_full[a]), 1); pbar_init(psmem_u32(&sm.acc_empty[a]), kEpiThreads / 32); }
+        sm.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {       // tensor memory: the whole of it, for two accumulators
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(psmem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tmem_fence_before();
+    __syncthreads();
+    tmem_fence_after();
+    const uint32_t tmem_base = sm.tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ loader
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+            uint32_t n = 0;
+            bool ok = true;
+#pragma unroll 1
+            for (int t = t_begin; t < t_end && ok; ++t) {
+                const int m = t / p.tiles_n, nn = t - m * p.tiles_n;
+#pragma unroll 1
+                for (int kb = 0; kb < k_blocks; ++kb, ++n) {
+                    const uint32_t s = n % kPStages, use = n / kPStages;
+                    if (use > 0 && !pbar_wait(psmem_u32(&sm.empty[s]), (use - 1) & 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t bar = psmem_u32(&sm.full[s]);
+                    pbar_expect_tx(bar, kStageA + kStageB);
+                    tma_load_2d(psmem_u32(sm.a[s]), &map_a, kb * kBK, m * kBM, bar);
+                    tma_load_2d(psmem_u32(sm.b[s]), &map_b, kb * kBK, nn * kBN, bar);
+                }
+            }
+            if (!ok) {     // winding down: let the loads already issued land before the CTA leaves
+                for (uint32_t f = n > kPStages ? n - kPStages : 0; f < n; ++f)
+                    for (uint32_t i = 0; i < 100000 && !pbar_try_wait(psmem_u32(&sm.full[f % kPStages]), (f / kPStages) & 1u); ++i) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t n = 0, tile_no = 0;
+            bool ok = true;
+#pragma unroll 1
+            for (int t = t_begin; t < t_end && ok; ++t, ++tile_no) {
+                const uint32_t acc = tile_no & 1u, acc_use = tile_no >> 1;
+                if (acc_use > 0 && !pbar_wait(psmem_u32(&sm.acc_empty[acc]), (acc_use - 1) & 1u, abort_flag)) { ok = false; break; }
+                tmem_fence_after();
+                const uint32_t d_addr = tmem_base + acc * kBN;
+#pragma unroll 1
+                for (int kb = 0; kb < k_blocks; ++kb, ++n) {
+                    const uint32_t s = n % kPStages, use = n / kPStages;
+                    if (!pbar_wait(psmem_u32(&sm.full[s]), use & 1u, abort_flag)) { ok = false; break; }
+                    tmem_fence_after();
+                    const uint64_t da = umma_desc_sw128(psmem_u32(sm.a[s])), db = umma_desc_sw128(psmem_u32(sm.b[s]));
+#pragma unroll
+                    for (int k4 = 0; k4 < kBK / 16; ++k4)      // 16 bf16 = 32 bytes further along the swizzled row
+                        umma_bf16(d_addr, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), (kb | k4) != 0 ? 1u : 0u);
+                    umma_commit(psmem_u32(&sm.empty[s]));       // the stage may be refilled when these are done
+                }
+                if (ok) umma_commit(psmem_u32(&sm.acc_full[acc]));
+            }
+        }
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------------ epilogue: thread t owns row t of the tile
+        const int et = tid - 128;                          // 0..127
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        float cref = kPNoRef, sum = 0.f, tau = neg_inf();
+        int n_list = 0;
+        bool lost = false;                 // a candidate found no room in the list: the piece cannot be trusted
+        int cur_m = -1;
+        bool ok = true;
+        uint32_t tile_no = 0;
+
+        auto compact = [&]() {         // raise tau to the K1-th largest entry of the list (to 16 bits) and drop what is below
+            if (n_list < p.K1) return;
+            uint32_t best = 0;         // the largest t, a multiple of 2^16, that at least K1 keys reach
+#pragma unroll 1
+            for (uint32_t bit = 0x80000000u; bit >= 0x00010000u; bit >>= 1) {
+                const uint32_t t = best | bit;
+                int cnt = 0;
+                for (int e = 0; e < n_list; ++e) cnt += sm.list_key[e][et] >= t;
+                if (cnt >= p.K1) best = t;
+            }
+            tau = best <= 0x007fffffu ? neg_inf() : unord32(best);
+            int kept = 0;
+            for (int e = 0; e < n_list; ++e) {
+                const uint32_t kx = sm.list_key[e][et];
+                const int c = sm.list_col[e][et];
+                if (kx >= best) { sm.list_key[kept][et] = kx; sm.list_col[kept][et] = c; ++kept; }
+            }
+            n_list = kept;
+        };
+        auto flush = [&](int m, int piece) {      // write this thread's piece of row m * kBM + et
+            compact();
+            const int row = m * kBM + et;
+            if (row < p.R) {
+                if (lost) atomicOr(p.status, kStatusOverflow);
+                const int64_t slot = (int64_t)row * p.pieces + piece;
+                p.out.ref[slot] = cref != kPNoRef ? __float2int_rn(cref) : INT_MIN;
+                p.out.sum[slot] = sum;
+                p.out.n[slot] = n_list;
+                for (int e = 0; e < n_list; ++e) {
+                    p.out.val[slot * kListCap + e] = unord32(sm.list_key[e][et]);
+                    p.out.col[slot * kListCap + e] = sm.list_col[e][et];
+                }
+            }
+        };
+        // piece of row block m that CTA c writes = c - (CTA that owns the row block's first tile)
+        auto first_cta = [&](int m) {
+            const long long t0 = (long long)m * p.tiles_n;
+            // largest c with c * n_tiles / grid <= t0
+            long long c = ((t0 + 1) * gridDim.x - 1) / n_tiles;
+            while (c > 0 && c * n_tiles / gridDim.x > t0) --c;
+            while ((c + 1) * n_tiles / gridDim.x <= t0) ++c;
+            return (int)c;
+        };
+
+#pragma unroll 1
+        for (int t = t_begin; t < t_end && ok; ++t, ++tile_no) {
+            const int m = t / p.tiles_n, nn = t - m * p.tiles_n;
+            if (m != cur_m) {
+                if (cur_m >= 0) flush(cur_m, (int)blockIdx.x - first_cta(cur_m));
+                cur_m = m;
+                cref = kPNoRef; sum = 0.f; tau = neg_inf(); n_list = 0; lost = false;
+            }
+            const uint32_t acc = tile_no & 1u, acc_use = tile_no >> 1;
+            if (!__all_sync(kFullMask, pbar_wait(psmem_u32(&sm.acc_full[acc]), acc_use & 1u, abort_flag))) { ok = false; break; }
+            tmem_fence_after();
+            const int col0 = nn * kBN;
+            const bool ragged = col0 + kBN > p.V;           // the vocabulary ends inside this tile
+#pragma unroll 1
+            for (int ch = 0; ch < kBN / 32; ++ch) {
+                float x[32];
+                tmem_ld32(tmem_base + lane_base + acc * kBN + ch * 32, x);
+                const int cbase = col0 + ch * 32;
+                if (ragged) {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) if (cbase + c >= p.V) x[c] = neg_inf();
+                }
+                float cm = x[0];
+#pragma unroll
+                for (int c = 1; c < 32; ++c) cm = fmaxf(cm, x[c]);
+                if (cm >= tau && cm != neg_inf()) {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (x[c] >= tau && x[c] != neg_inf()) {
+                            if (n_list < kListCap) { sm.list_key[n_list][et] = ord32(x[c]); sm.list_col[n_list][et] = cbase + c; ++n_list; }
+                            else lost = true;
+                        }
+                }
+                // the normaliser
+                const float need = cm * kPLog2e;
+                if (need > cref + 8.f) {
+                    const float cn = ceilf(need);
+                    const float dd = cref - cn;
+                    sum *= dd < -126.f ? 0.f : ppow2i((int)dd);
+                    cref = cn;
+                }
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                for (int c = 0; c < 32; c += 4) {
+                    s0 += pex2(fmaf(x[c], kPLog2e, -cref)); s1 += pex2(fmaf(x[c + 1], kPLog2e, -cref));
+                    s2 += pex2(fmaf(x[c + 2], kPLog2e, -cref)); s3 += pex2(fmaf(x[c + 3], kPLog2e, -cref));
+                }
+                sum += (s0 + s1) + (s2 + s3);
+                // room for the next 32 columns in every list of the warp, or everybody tidies up now
+                if (__any_sync(kFullMask, n_list > kListCap - 32)) compact();
+            }
+            // the accumulator may be overwritten
+            tmem_fence_before();
+            __syncwarp();
+            if (lane == 0) pbar_arrive(psmem_u32(&sm.acc_empty[acc]));
+        }
+        if (ok && cur_m >= 0) flush(cur_m, (int)blockIdx.x - first_cta(cur_m));
+    }
+    tmem_fence_before();
+    __syncthreads();
+    tmem_fence_after();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    if (tid == 0 && sm.abort_flag) atomicOr(p.status, kStatusTimeout);
+}
+
+// Orders the pieces of every row exactly: one warp per row gathers the candidates of the row's pieces, ranks them
+// (value descending, lower index first) and writes the K1 best and the row's normaliser.
+__global__ void project_merge_kernel(ProjParams p, int grid_scan, RowTop top) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= p.R) return;
+    const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
+    const int m = row / kBM;
+    // CTAs that own the first and the last tile of this row block
+    auto owner = [&](long long t) {
+        long long c = ((t + 1) * grid_scan - 1) / n_tiles;
+        while (c > 0 && c * n_tiles / grid_scan > t) --c;
+        while ((c + 1) * n_tiles / grid_scan <= t) ++c;
+        return (int)c;
+    };
+    const int c0 = owner((long long)m * p.tiles_n), c1 = owner((long long)(m + 1) * p.tiles_n - 1);
+    const int n_pieces = c1 - c0 + 1;
+    const int64_t base = (int64_t)row * p.pieces;
+    // normaliser: pieces in order
+    if (lane == 0) {
+        int C = INT_MIN;
+        for (int g = 0; g < n_pieces; ++g) C = max(C, p.out.ref[base + g]);
+        float total = 0.f;
+        if (C != INT_MIN)
+            for (int g = 0; g < n_pieces; ++g)
+                if (p.out.ref[base + g] != INT_MIN) total += p.out.sum[base + g] * ppow2i(p.out.ref[base + g] - C);
+        float lse = neg_inf();
+        if (C != INT_MIN && total > 0.f) {
+            constexpr float kLn2Hi = 0.693147182464599609375f, kLn2Lo = -1.904654299957767e-9f;
+            const float c = (float)C, hi = c * kLn2Hi, lo = fmaf(c, kLn2Hi, -hi) + c * kLn2Lo;
+            lse = hi + (logf(total) + lo);
+        }
+        top.lse[row] = lse;
+    }
+    // candidates: entry e of piece g; rank by counting the better ones
+    float* tv = top.val + (int64_t)row * p.K1;
+    int32_t* ti = top.idx + (int64_t)row * p.K1;
+    int total_n = 0;
+    for (int g = 0; g < n_pieces; ++g) total_n += p.out.n[base + g];
+    for (int e = total_n + lane; e < p.K1; e += 32) { tv[e] = neg_inf(); ti[e] = -1; }
+    for (int g = 0; g < n_pieces; ++g) {
+        const int ng = p.out.n[base + g];
+        for (int e = lane; e < ng; e += 32) {
+            const float x = p.out.val[(base + g) * kListCap + e];
+            const int w = p.out.col[(base + g) * kListCap + e];
+            const uint64_t key = row_key(x, w);
+            int rank = 0;
+            for (int g2 = 0; g2 < n_pieces; ++g2) {
+                const int n2 = p.out.n[base + g2];
+                for (int e2 = 0; e2 < n2; ++e2)
+                    rank += row_key(p.out.val[(base + g2) * kListCap + e2], p.out.col[(base + g2) * kListCap + e2]) > key;
+            }
+            if (rank < p.K1) { tv[rank] = x; ti[rank] = w; }
+        }
+    }
+}
+
+// One warp per (row, constraint position of the row's sentence): the inner product, fp32, lanes striding over D.
+__global__ void constraint_logits_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t hs, const __nv_bfloat16* __restrict__ embed,
+                                         int64_t es, int D, int R, int k, const SentCons* __restrict__ cons, float* __restrict__ out) {
+    const int64_t gw = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    const int r = (int)(gw >> 6), j = (int)(gw & 63);
+    if (r >= R) return;
+    const SentCons& sc = cons[r / k];
+    if (j >= sc.C) return;
+    const __nv_bfloat16* h = hidden + (int64_t)r * hs;
+    const __nv_bfloat16* e = embed + (int64_t)sc.ctok[j] * es;
+    float acc = 0.f;
+    for (int i = lane; i < D; i += 32) acc = fmaf(load_logit<__nv_bfloat16>(h + i), load_logit<__nv_bfloat16>(e + i), acc);
+    acc = warp_sum(acc);
+    if (lane == 0) out[(int64_t)r * kMaxC + j] = acc;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)f;
+    }
+    return fn;
+}
+
+// [rows, D] bf16 row-major, rows `stride` elements apart: boxes of 64 elements x box_rows rows, 128-byte swizzle,
+// zero fill beyond the edges
+bool make_map(CUtensorMap* map, const void* base, int rows, int D, int64_t stride, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)stride * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t launch_constraint_logits(const void* hidden, int64_t hidden_stride, const void* embed, int64_t embed_stride,
+                                     int D, const Dims& d, const SentCons* cons, float* out, cudaStream_t st, int* launches) {
+    const int64_t warps = (int64_t)d.R * kMaxC;
+    const int per_block = 8;
+    constraint_logits_kernel<<<(unsigned)((warps + per_block - 1) / per_block), per_block * 32, 0, st>>>(
+        (const __nv_bfloat16*)hidden, hidden_stride, (const __nv_bfloat16*)embed, embed_stride, D, d.R, d.k, cons, out);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+int project_pieces(int R, int V, int sm_count) {
+    const int tiles_m = (R + kBM - 1) / kBM, tiles_n = (V + kBN - 1) / kBN;
+    const long long n_tiles = (long long)tiles_m * tiles_n;
+    const int grid = (int)(n_tiles < sm_count ? n_tiles : sm_count);
+    return (grid + tiles_m - 1) / tiles_m + 2;
+}
+
+int project_list_cap() { return kListCap; }
+
+bool project_scan_usable(const void* hidden, int64_t hidden_stride, const void* embed, int64_t embed_stride, int D, int K1) {
+    if (((uintptr_t)hidden & 15u) || ((uintptr_t)embed & 15u) || ((hidden_stride * 2) & 15) || ((embed_stride * 2) & 15)) return false;
+    return D >= 8 && D % 8 == 0 && K1 <= 32;
+}
+
+cudaError_t configure_project_scan() {
+    return cudaFuncSetAttribute(project_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ProjSmem) + 1024);
+}
+
+cudaError_t launch_project_scan(const void* hidden, int64_t hidden_stride, const void* embed, int64_t embed_stride,
+                                int R, int V, int D, int K1, const ProjPieces& pieces, int piece_stride,
+                                const RowTop& top, uint32_t* status, int sm_count, cudaStream_t st, int* launches) {
+    CUtensorMap map_a, map_b;
+    if (!make_map(&map_a, hidden, R, D, hidden_stride, kBM) || !make_map(&map_b, embed, V, D, embed_stride, kBN))
+        return cudaErrorInvalidValue;
+    ProjParams p;
+    p.R = R; p.V = V; p.D = D; p.K1 = K1;
+    p.tiles_m = (R + kBM - 1) / kBM; p.tiles_n = (V + kBN - 1) / kBN;
+    p.pieces = piece_stride; p.out = pieces; p.status = status;
+    const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
+    const int grid = (int)(n_tiles < sm_count ? n_tiles : sm_count);
+    project_scan_kernel<<<grid, kProjThreads, sizeof(ProjSmem) + 1024, st>>>(map_a, map_b, p);
+    ++*launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int warps = 8;
+    project_merge_kernel<<<(R + warps - 1) / warps, warps * 32, 0, st>>>(p, grid, top);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace dba

@@ -1,5 +1,6 @@
-// Row scan: per (row, segment) the reference maximum, sum of exponentials and the K1 largest entries.
-// This file holds the generic kernel (any alignment, plain loads) and the stand-alone merge kernel.
+// Row scan: per row the log-sum-exp and the K1 largest entries.
+// This file holds the generic kernel (any alignment, plain loads), the choice between it and the streaming one,
+// segment planning, and the stand-alone merge of the streaming kernel's per-segment results.
 #include "dba_device.cuh"
 #include "dba_internal.h"
 
@@ -7,7 +8,7 @@ namespace dba {
 
 namespace {
 
-constexpr int kScanThreads = 256;
+constexpr int kScanThreads = 512;
 
 // Deterministic block reductions over kScanThreads threads (fixed tree, result broadcast to all).
 __device__ float block_max(float v, float* sm) {
@@ -38,45 +39,42 @@ __device__ uint64_t block_max_u64(uint64_t v, uint64_t* sm) {
     return r;
 }
 
-// Generic scan: one CTA per (row, segment); K1 + 2 passes over the segment (it stays in L2).
+// Generic scan: one CTA per row; K1 + 2 passes over the row (it stays in L2 between them).
 template <typename T>
 __global__ void __launch_bounds__(kScanThreads)
-row_scan_generic_kernel(const T* __restrict__ logits, int64_t stride, int V, int S, int seg_len, int K1,
-                        int eos, const float* __restrict__ open_score, const int32_t* __restrict__ open_token,
-                        int32_t* __restrict__ zero_count, float* __restrict__ part_m, float* __restrict__ part_s,
+row_scan_generic_kernel(const T* __restrict__ logits, int64_t stride, int V, int K1, int eos,
+                        const float* __restrict__ open_score, const int32_t* __restrict__ open_token,
+                        int32_t* __restrict__ zero_count, float* __restrict__ row_lse,
                         float* __restrict__ top_val, int32_t* __restrict__ top_idx) {
     __shared__ float smf[kScanThreads / 32];
     __shared__ uint64_t smu[kScanThreads / 32];
-    const int item = blockIdx.x;
-    if (zero_count && item == 0 && threadIdx.x == 0) *zero_count = 0;
-    const int r = item / S, g = item - r * S;
+    const int r = blockIdx.x;
+    if (zero_count && r == 0 && threadIdx.x == 0) *zero_count = 0;
     if (open_score) {
         if (open_score[r] == neg_inf() || open_token[r] == eos) return;   // empty or finished slot
     }
-    const int lo = g * seg_len;
-    const int hi = min(V, lo + seg_len);
     const T* row = logits + (int64_t)r * stride;
 
     float m = neg_inf();
-    for (int w = lo + threadIdx.x; w < hi; w += kScanThreads) m = fmaxf(m, load_logit<T>(row + w));
+    for (int w = threadIdx.x; w < V; w += kScanThreads) m = fmaxf(m, load_logit<T>(row + w));
     m = block_max(m, smf);
     float s = 0.f;
     if (m != neg_inf())
-        for (int w = lo + threadIdx.x; w < hi; w += kScanThreads) s += expf(load_logit<T>(row + w) - m);
+        for (int w = threadIdx.x; w < V; w += kScanThreads) s += expf(load_logit<T>(row + w) - m);
     s = block_sum(s, smf);
-    if (threadIdx.x == 0) { part_m[item] = m; part_s[item] = s; }
+    if (threadIdx.x == 0) row_lse[r] = m == neg_inf() ? neg_inf() : m + logf(s);
 
     uint64_t prev = ~0ull;
     for (int i = 0; i < K1; ++i) {
         uint64_t best = 0;
-        for (int w = lo + threadIdx.x; w < hi; w += kScanThreads) {
+        for (int w = threadIdx.x; w < V; w += kScanThreads) {
             uint64_t key = row_key(load_logit<T>(row + w), w);
             if (key < prev && key > best) best = key;
         }
         best = block_max_u64(best, smu);
         if (threadIdx.x == 0) {
-            top_val[(int64_t)item * K1 + i] = best ? row_key_val(best) : neg_inf();
-            top_idx[(int64_t)item * K1 + i] = best ? row_key_idx(best) : -1;
+            top_val[(int64_t)r * K1 + i] = best ? row_key_val(best) : neg_inf();
+            top_idx[(int64_t)r * K1 + i] = best ? row_key_idx(best) : -1;
         }
         prev = best ? best : 0;   // once exhausted, nothing is below key 0
     }
@@ -115,7 +113,22 @@ __global__ void row_merge_kernel(int R, int S, int K1, int n_top, const float* _
     }
 }
 
+// The stand-alone scan has no handle whose later calls could report a failed wait: if the scan recorded one,
+// every row's result is replaced by one that cannot be taken for a real one (normaliser NaN, list (-inf, -1)).
+__global__ void scan_check_kernel(const uint32_t* __restrict__ status, int R, int n_top, RowTop top) {
+    if (!(*status & (kStatusTimeout | kStatusOverflow))) return;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < (int64_t)R * n_top; i += (int64_t)gridDim.x * blockDim.x) {
+        top.val[i] = neg_inf(); top.idx[i] = -1;
+        if (i < R) top.lse[i] = __int_as_float(0x7fc00000);
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_scan_check(const uint32_t* status, int R, int n_top, const RowTop& top, cudaStream_t st) {
+    scan_check_kernel<<<64, 256, 0, st>>>(status, R, n_top, top);
+    return cudaGetLastError();
+}
 
 void plan_segments(Dims& d, int sm_count) {
     // Segments are whole 4 KB chunks, at most eleven of them (what one team of the streaming kernel holds);
@@ -148,28 +161,28 @@ int max_segments(int V, int dtype) {
 
 cudaError_t launch_row_scan(const void* logits, int64_t stride, const Dims& d, const float* open_score,
                             const int32_t* open_token, const int32_t* open_list, const int32_t* open_count,
-                            int32_t* zero_count, const ScanOut& out, uint32_t* status, int sm_count, cudaStream_t st,
-                            int* launches) {
+                            int32_t* zero_count, const RowTop& out, const ScanScratch& part, uint32_t* status,
+                            int sm_count, const ScanDebug& dbg, cudaStream_t st, int* launches, bool* partial) {
     ++*launches;
-    if (row_scan_tma_usable(logits, stride, d))
-        return launch_row_scan_tma(logits, stride, d, open_list, open_count, zero_count, out, status, sm_count, st);
-    const int items = d.R * d.S;
+    *partial = row_scan_tma_usable(logits, stride, d);
+    if (*partial)
+        return launch_row_scan_tma(logits, stride, d, open_list, open_count, zero_count, part, status, sm_count, dbg, st);
     if (d.dtype == DBA_F32)
-        row_scan_generic_kernel<float><<<items, kScanThreads, 0, st>>>(
-            (const float*)logits, stride, d.V, d.S, d.seg_len, d.K1, d.eos_id, open_score, open_token, zero_count,
-            out.m, out.s, out.top_val, out.top_idx);
+        row_scan_generic_kernel<float><<<d.R, kScanThreads, 0, st>>>(
+            (const float*)logits, stride, d.V, d.K1, d.eos_id, open_score, open_token, zero_count, out.lse, out.val,
+            out.idx);
     else
-        row_scan_generic_kernel<__nv_bfloat16><<<items, kScanThreads, 0, st>>>(
-            (const __nv_bfloat16*)logits, stride, d.V, d.S, d.seg_len, d.K1, d.eos_id, open_score, open_token,
-            zero_count, out.m, out.s, out.top_val, out.top_idx);
+        row_scan_generic_kernel<__nv_bfloat16><<<d.R, kScanThreads, 0, st>>>(
+            (const __nv_bfloat16*)logits, stride, d.V, d.K1, d.eos_id, open_score, open_token, zero_count, out.lse,
+            out.val, out.idx);
     return cudaGetLastError();
 }
 
-cudaError_t launch_row_merge(const Dims& d, const ScanOut& part, int n_top, float* row_lse, float* top_val,
+cudaError_t launch_row_merge(const Dims& d, const ScanScratch& part, int n_top, float* row_lse, float* top_val,
                              int32_t* top_idx, cudaStream_t st, int* launches) {
     const int warps = 4;
     row_merge_kernel<<<(d.R + warps - 1) / warps, warps * 32, 0, st>>>(d.R, d.S, d.K1, n_top, part.m, part.s,
-                                                                      part.top_val, part.top_idx, row_lse,
+                                                                      part.val, part.idx, row_lse,
                                                                       top_val, top_idx);
     ++*launches;
     return cudaGetLastError();

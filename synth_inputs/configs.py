@@ -98,7 +98,7 @@ def _constraints(cfg_id, B, V, rng, C_fixed=None):
             cons.append(_split(_distinct_ids(rng, total, V), lens))
         elif cfg_id == 4:
             ids = _distinct_ids(rng, C_fixed, V); cons.append([[i] for i in ids])
-        elif cfg_id == 5:
+        elif cfg_id in (5, 6):
             lens = _composition(rng, 10, 1, 4, 10)
             cons.append(_split(_distinct_ids(rng, 10, V), lens))
         else:
@@ -112,6 +112,9 @@ CONFIGS = {
     "ragged":  dict(cfg_id=3, B=64,  k=10, V=32000, steps=80,  dtype="bf16", zipf=True,  boost=True),
     "scaling": dict(cfg_id=4, B=16,  k=20, V=32000, steps=100, dtype="f32",  zipf=True,  boost=True),
     "serving": dict(cfg_id=5, B=256, k=20, V=64000, steps=120, dtype="bf16", zipf=True,  boost=True),
+    # not one of the five named configurations: a second shape for the long-row path (a Transformer-sized
+    # vocabulary in fp32: rows of 512 KB), constraints as in "serving"
+    "transformer": dict(cfg_id=6, B=128, k=20, V=131072, steps=40, dtype="f32", zipf=True, boost=True),
 }
 
 

@@ -59,7 +59,7 @@ def lockstep(wl, stepper, steps=None, threads=8, gpu_gen=None, lse_tol=1e-5, fla
     larger than any logit (a read past the end of a row would win every selection)."""
     import torch
     steps = wl.steps if steps is None else steps
-    orc = O.Batch(wl.k, wl.V, steps, wl.constraints, flags=flags & 3, threads=threads, prune=prune)
+    orc = O.Batch(wl.k, wl.V, steps, wl.constraints, flags=flags & 11, threads=threads, prune=prune)
     host_gen = LogitStream(wl) if gpu_gen is None else None
     worst = 0.0
     for t in range(steps):
@@ -115,9 +115,10 @@ def check_beam_invariants(g, wl, C_per_sentence, where):
 def free_run(wl, stepper, sample, steps, gpu_gen, threads=8, score_tol=1e-5):
     """The CUDA library in its own closed loop over the whole workload (its own normalisers, logits generated
     from its own beam), next to independent oracle runs of the sampled sentences.  Sentences must match
-    exactly; where a sampled sentence first differs, the two beams must hold the same scores rank by rank
-    within the accumulated tolerance (a tie decided by the last bit of a normaliser), and the sentence leaves
-    the comparison.  Returns (compared sentence-steps, sentences that left)."""
+    exactly.  Where a sampled sentence first differs, the difference must be a tie decided by the last bits of
+    a normaliser: the two beams hold the same scores rank by rank within the accumulated tolerance, and at the
+    first differing slot the oracle's own candidates hold another score within that tolerance (the near-tie);
+    the sentence then leaves the comparison.  Returns (compared sentence-steps, [(step, sentence) that left])."""
     import torch
     sub = wl.subset(sample)
     orc = O.Batch(sub.k, sub.V, steps, sub.constraints, threads=threads)
@@ -127,7 +128,7 @@ def free_run(wl, stepper, sample, steps, gpu_gen, threads=8, score_tol=1e-5):
     tok = torch.full((wl.R,), 0, dtype=torch.int32, device="cuda"); tok[::k] = 1
     mask = torch.zeros(wl.R, dtype=torch.int64, device="cuda")
     alive = [True] * len(sample)
-    compared = 0
+    compared, departures = 0, []
     for t in range(steps):
         x_dev = gpu_gen.step_logits(t, tok, mask)
         out = stepper.step(x_dev)
@@ -149,6 +150,13 @@ def free_run(wl, stepper, sample, steps, gpu_gen, threads=8, score_tol=1e-5):
                 f"step {t} sentence {b}: scores differ beyond {tol}"
             if all((gs[f] == os_[f]).all() for f in BEAM_FIELDS):
                 compared += 1
-            else:
-                alive[i] = False
-    return compared, alive.count(False)
+                continue
+            # the first differing slot must sit at a near-tie among the oracle's candidates of this step
+            slot = int(np.nonzero(~np.all([gs[f] == os_[f] for f in BEAM_FIELDS], axis=0))[0][0])
+            cand = np.sort(orc.sent[i].candidates()["score"].astype(np.float64))
+            here = float(os_["score"][slot])
+            near = np.abs(cand - here) <= tol
+            assert near.sum() >= 2, f"step {t} sentence {b} slot {slot}: selections differ without a tie to explain it"
+            alive[i] = False
+            departures.append((t, b))
+    return compared, departures

@@ -127,6 +127,94 @@ def test_repeated_scans_of_the_same_rows_agree(dba, dtype):
         assert abs(float(lse[r]) - O.row_lse(row_in)) <= 1e-5
 
 
+# ------------------------------------------------------------------------------------------ fused projection
+@pytest.mark.parametrize("R,V,D,n_top", [(5, 1000, 64, 7), (128, 4096, 256, 22), (300, 20011, 128, 22), (20, 64000, 1024, 22),
+                                          (131, 5000, 72, 32), (260, 33000, 64, 12)])
+def test_fused_projection_and_row_scan_match_the_oracle(dba, R, V, D, n_top):
+    """Section 2's output projection on the tensor cores with the row scan in its epilogue, against the oracle's
+    double-precision inner products.  The kernel accumulates bf16 products in fp32, so a logit may differ from
+    the oracle's by the rounding of D additions: normalisers within 1e-4, listed values within 1e-4 rank by rank,
+    and where the listed word differs from the oracle's it must be one whose exact logit ties with the oracle's
+    choice within that bound."""
+    from synth_inputs.logits import to_bf16_bits
+    rng = np.random.default_rng(R + V + D)
+    h = rng.normal(0, 1, (R, D)).astype(np.float32)
+    mu = (-1.1 * np.log(rng.permutation(V) + 1.0)).astype(np.float32)          # Zipf-shaped word offsets
+    e = rng.normal(0, 1, (V, D)).astype(np.float32) / np.float32(np.sqrt(D))
+    e[:, 0] = mu; h[:, 0] = 1.0                                                  # logits = offset + noise
+    hb, eb = to_bf16_bits(h), to_bf16_bits(e)
+    X = O.project(hb, eb)
+    hd = torch.from_numpy(hb.view(np.int16)).cuda().view(torch.bfloat16)
+    ed = torch.from_numpy(eb.view(np.int16)).cuda().view(torch.bfloat16)
+    lse, val, idx = dba.project_scan(hd, ed, n_top)
+    lse, val, idx = lse.cpu().numpy(), val.cpu().numpy(), idx.cpu().numpy()
+    tol = 1e-4
+    for r in range(R):
+        assert abs(float(lse[r]) - O.row_lse(X[r])) <= tol, (r, lse[r], O.row_lse(X[r]))
+        wv, wi = O.row_top(X[r], n_top)
+        assert np.abs(val[r] - wv).max() <= tol, (r, val[r], wv)
+        assert ((idx[r] >= 0) & (idx[r] < V)).all() and len(set(idx[r].tolist())) == n_top
+        assert np.abs(X[r][idx[r]] - wv).max() <= tol, (r, idx[r], wi)
+
+
+def test_fused_step_follows_the_oracle_on_the_projected_logits(dba):
+    """dba_step_fused against the oracle stepping on the exactly projected logits.  Sentences must match field by
+    field; where one first differs the two beams must hold the same scores rank by rank within the accumulated
+    tolerance of the fp32 accumulation (a near-tie decided the other way), and it leaves the comparison."""
+    from synth_inputs.logits import to_bf16_bits
+    from tests.parity import BEAM_FIELDS
+    B, k, V, D, steps = 6, 5, 3000, 64, 16
+    cons = [[[5, 6]], [[7], [8, 9]], [], [[10]], [[11, 12, 13]], [[14], [15]]]
+    rng = np.random.default_rng(42)
+    mu = (-1.1 * np.log(rng.permutation(V) + 1.0)).astype(np.float32)
+    e = rng.normal(0, 1, (V, D)).astype(np.float32) / np.float32(np.sqrt(D))
+    e[:, 0] = mu
+    e[:, 1] = 0.0; e[2, 1] = 1.0                     # the end token's logit follows hidden[:, 1]
+    for c in cons:                                   # constraint tokens are likely words
+        for ph in c:
+            for w in ph:
+                e[w, 0] = -1.0
+    eb = to_bf16_bits(e)
+    ed = torch.from_numpy(eb.view(np.int16)).cuda().view(torch.bfloat16)
+    st = dba.DbaStepper(B, k, V, steps, constraints=cons, dtype=dba.F32, flags=dba.FLAG_FUSED_PROJECTION)
+    orc = O.Batch(k, V, steps, cons, threads=1)
+    alive = [True] * B
+    compared = 0
+    for t in range(steps):
+        h = rng.normal(0, 1, (B * k, D)).astype(np.float32)
+        h[:, 0] = 1.0
+        h[:, 1] = -6.0 if t < 8 else 4.0             # the end token becomes likely in the second half
+        hb = to_bf16_bits(h)
+        X = O.project(hb, eb)
+        orc.step(X)
+        out = st.step_fused(torch.from_numpy(hb.view(np.int16)).cuda().view(torch.bfloat16), ed)
+        g, ob = gpu_beam(out), orc.beam()
+        tol = 1e-4 * (t + 1)
+        for b in range(B):
+            if not alive[b]:
+                continue
+            sl = slice(b * k, (b + 1) * k)
+            fin = np.isfinite(ob["score"][sl])
+            assert (np.isfinite(g["score"][sl]) == fin).all()
+            assert np.abs(g["score"][sl][fin] - ob["score"][sl][fin]).max(initial=0) <= tol, (t, b)
+            if all((g[f][sl] == ob[f][sl]).all() for f in BEAM_FIELDS):
+                compared += 1
+            else:
+                alive[b] = False
+        if t > 0 and not any(alive):
+            break
+        # both sides go on from the oracle's beam only while they agree; a sentence that left is not looked at again
+    assert sum(alive) >= B - 2 and compared >= (B - 2) * steps
+    assert st.counters()[1] == 0
+    tokens, length, score, flags = st.finalize()
+    done = [d for _, _, d in orc.finalize()]
+    for b in range(B):
+        if alive[b]:
+            assert bool(flags[b] & 1) == done[b]
+    assert sum(done) >= 3
+    st.close()
+
+
 # ------------------------------------------------------------------------------------------ whole step
 def test_step_parity_tiny(dba):
     wl = make_workload("tiny")
@@ -154,8 +242,8 @@ def test_step_parity_ragged(dba):
 def test_step_parity_scaling(dba, C):
     from synth_inputs.gpu import GpuLogitStream
     wl = make_workload("scaling", C=C)
-    st = _stepper(dba, wl, steps=40)
-    orc, worst = lockstep(wl, st, steps=40, gpu_gen=GpuLogitStream(wl))
+    st = _stepper(dba, wl)
+    orc, worst = lockstep(wl, st, gpu_gen=GpuLogitStream(wl))        # all 100 steps
     assert_finalize_equal(st, orc)
 
 
@@ -175,9 +263,27 @@ def test_serving_full_size_free_run_against_sampled_oracle(dba):
     from tests.parity import free_run
     wl = make_workload("serving")
     st = _stepper(dba, wl)
-    steps = 30
-    compared, left = free_run(wl, st, [3, 77, 140, 201, 254], steps, GpuLogitStream(wl))
-    assert left <= 1 and compared >= 4 * steps
+    steps = wl.steps           # all 120: finished rows, the shrinking list of open rows and the last waves included
+    sample = [3, 40, 77, 111, 140, 201, 230, 254]
+    compared, left = free_run(wl, st, sample, steps, GpuLogitStream(wl))
+    assert len(left) <= 1 and compared >= (len(sample) - 1) * steps, left     # a departure is a verified near-tie
+    assert st.counters()[0] == 0
+    tokens, length, score, flags = st.finalize()
+    assert (flags & 1).sum() >= 200                       # the stream lets most sentences finish
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("phrasal", {}), ("ragged", {}), ("scaling", dict(C=1)),
+                                     ("scaling", dict(C=50))])
+def test_small_workloads_free_running_on_the_gpus_own_normalisers(dba, name, kw):
+    """The four small configurations, every sentence, every step, with the library ranking by the normalisers it
+    computes itself (the lock-step tests hand it the oracle's)."""
+    from synth_inputs.gpu import GpuLogitStream
+    from tests.parity import free_run
+    wl = make_workload(name, **kw)
+    st = _stepper(dba, wl)
+    compared, left = free_run(wl, st, list(range(wl.B)), wl.steps, GpuLogitStream(wl))
+    assert len(left) <= max(1, wl.B // 16) and compared >= (wl.B - len(left) - 1) * wl.steps, left
+    st.close()
 
 
 @pytest.mark.parametrize("dtype,B,V", [("f32", 210, 262144), ("bf16", 212, 524288)])
@@ -192,7 +298,7 @@ def test_logit_matrices_beyond_four_gigabytes(dba, dtype, B, V):
     steps = 5
     sample = [0, B // 2, B - 5, B - 1]
     compared, left = free_run(wl, st, sample, steps, GpuLogitStream(wl))
-    assert left <= 1 and compared >= 3 * steps
+    assert len(left) <= 1 and compared >= 3 * steps
 
 
 # ------------------------------------------------------------------------------------------ edge cases
@@ -330,6 +436,20 @@ def test_threshold_pruning_and_stop_bits_match_the_oracle(dba, name, kw, theta):
     st.close()
 
 
+@pytest.mark.parametrize("name,kw,theta", [("ragged", dict(B=6, V=4096, steps=40), 2.0), ("ragged", dict(B=6, V=4096, steps=40), 0.5),
+                                           ("serving", dict(B=3, V=8192, steps=60), 1.0)])
+def test_pruning_by_normalised_completed_scores_matches_the_oracle(dba, name, kw, theta):
+    """Section 4's other reading: completed hypotheses enter the threshold comparison with score / length.  The
+    hypotheses removed are then not always the tail of the beam."""
+    wl = make_workload(name, **kw)
+    st = dba.DbaStepper(wl.B, wl.k, wl.V, wl.steps, constraints=wl.constraints,
+                        dtype=dba.BF16 if wl.dtype == "bf16" else dba.F32, prune=theta, flags=dba.FLAG_PRUNE_NORMALISED)
+    orc, worst = lockstep(wl, st, prune=theta, flags=dba.FLAG_PRUNE_NORMALISED)
+    assert_finalize_equal(st, orc)
+    assert (orc.stop_flags() & 2).any()
+    st.close()
+
+
 @pytest.mark.parametrize("flags", [1, 2, 3])
 def test_flags_adjust_off_and_length_norm(dba, flags):
     wl = make_workload("ragged", B=6, V=3000, steps=50)
@@ -455,6 +575,38 @@ def test_step_host_equals_step_and_reset_replays(dba):
     with pytest.raises(dba.DbaError) as e:
         a.step(to_device_logits(trace[0][0], wl))
     assert e.value.code == 3                                        # DBA_ERR_STATE: past max_steps
+
+
+def test_a_device_wait_that_runs_out_is_reported_and_the_device_stays_usable(dba):
+    """Failure detection without a fault: the row scan's waits are bounded.  The testing aid makes every warp
+    announce its first copy without issuing it and shortens the limit to about a millisecond: the waits run out,
+    the kernel records that and returns, dba_finalize reports DBA_ERR_TIMEOUT.  A fresh handle on the same
+    device and stream then steps in parity with the oracle.  The stand-alone scan reports the same failure in
+    its results (NaN normalisers, empty lists)."""
+    wl = make_workload("ragged", B=4, V=8192, steps=6)
+    gen = LogitStream(wl)
+    tok = np.zeros(wl.R, np.int32); tok[::wl.k] = 1
+    x = to_device_logits(gen.step_logits(0, tok, np.zeros(wl.R, np.uint64)), wl)
+    st = _stepper(dba, wl)
+    st.test_hook(wait_clocks=2_000_000, drop_item=0)
+    st.step(x)                                   # enqueued; the failure is on the device
+    with pytest.raises(dba.DbaError) as e:
+        st.finalize()
+    assert e.value.code == 5                     # DBA_ERR_TIMEOUT
+    st.close()
+    L = dba.lib()
+    try:
+        assert L.dba_test_hook(None, 2_000_000, 0) == 0
+        lse, val, idx = dba.row_scan(x, 5)
+        assert torch.isnan(lse).all() and (idx == -1).all() and torch.isinf(val).all()
+    finally:
+        assert L.dba_test_hook(None, 0, -1) == 0
+    lse, val, idx = dba.row_scan(x, 5)
+    assert torch.isfinite(lse).all() and (idx >= 0).all()
+    st2 = _stepper(dba, wl)
+    orc, worst = lockstep(wl, st2)
+    assert_finalize_equal(st2, orc)
+    st2.close()
 
 
 def test_argument_errors_are_reported_not_launched(dba):
