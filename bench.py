@@ -41,6 +41,10 @@ def parse():
     ap.add_argument("--stream-steps", type=int, default=None, help="keep only the first steps of the stream resident")
     ap.add_argument("--e2e-steps", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fused", action="store_true",
+                    help="the step fused into the output projection (dba_step_fused): hidden states and embedding in, "
+                         "logits never materialised; reports a tensor-core roofline")
+    ap.add_argument("--D", type=int, default=1024, help="hidden size of the fused step")
     return ap.parse_args()
 
 
@@ -49,6 +53,14 @@ def measured_peak():
     if os.path.exists(p):
         return float(json.load(open(p))["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def measured_tensor_peak():
+    """Dense bf16 TFLOP/s of a cuBLAS GEMM loop under the power cap (the kernel is timed inside a long step)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["bf16_tflops_sustained"]), "measured, sustained"
+    return 1400.0, "fallback, sustained"
 
 
 def ncu_traffic(workload, open_rows_per_launch):
@@ -350,10 +362,105 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_fused(args):
+    """dba_step_fused on the workload's shape: synthetic hidden states [R, D] and output embedding [V, D] (bf16,
+    Zipf-shaped word offsets in one embedding column, an end-token column that rises along the stream), one GPU."""
+    import torch
+    import paper_1804_06609_b200 as pkg
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    wl = workload_of(args)
+    D, R, V = args.D, wl.R, wl.V
+    g = torch.Generator(device=dev); g.manual_seed(wl.seed)
+    e = torch.randn(V, D, device=dev, generator=g) / D ** 0.5
+    e[:, 0] = -1.1 * torch.log(torch.randperm(V, device=dev, generator=g).float() + 1.0)
+    e[:, 1] = 0.0; e[2, 1] = 1.0
+    for c in wl.constraints:
+        for ph in c:
+            e[ph, 0] = 1.0                     # constraint tokens are likely words: the constraints get met
+    embed = e.to(torch.bfloat16)
+    T = min(wl.steps, 32)
+    hidden = torch.randn(T, R, D, device=dev, generator=g)
+    hidden[:, :, 0] = 1.0
+    hidden[:, :, 1] = torch.linspace(-8.0, 10.0, T, device=dev)[:, None]
+    hidden = hidden.to(torch.bfloat16)
+    st = pkg.DbaStepper(wl.B, wl.k, V, wl.steps, constraints=wl.constraints, dtype=pkg.F32, device=dev,
+                        flags=pkg.FLAG_FUSED_PROJECTION)
+
+    def replay(n, start=0):
+        for i in range(start, start + n):
+            if i % T == 0:
+                st.reset()
+            st.step_fused(hidden[i % T], embed)
+
+    replay(args.warmup)
+    launches0 = st.launch_count()
+    sampler = ClockSampler(0); sampler.start()
+    time.sleep(0.05)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    e0.record()
+    replay(args.steps, start=args.warmup)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    sampler.stop_flag = True; sampler.join()
+    ms = e0.elapsed_time(e1)
+    launches = st.launch_count() - launches0
+    st.timing_enable(True)
+    replay(args.steps, start=args.warmup + args.steps)
+    kt, ksteps = st.timing_read()
+    st.timing_enable(False)
+    tokens, length, score, flags = st.finalize()
+    # for comparison, the same work unfused: a library GEMM that writes the logits (bf16), then the step on them
+    st2 = pkg.DbaStepper(wl.B, wl.k, V, wl.steps, constraints=wl.constraints, dtype=pkg.BF16, device=dev)
+    logits = torch.empty(R, V, dtype=torch.bfloat16, device=dev)
+    embed_t = embed.t()
+
+    def replay_unfused(n, start=0):
+        for i in range(start, start + n):
+            if i % T == 0:
+                st2.reset()
+            torch.matmul(hidden[i % T], embed_t, out=logits)
+            st2.step(logits)
+
+    replay_unfused(args.warmup)
+    torch.cuda.synchronize(dev)
+    u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    u0.record()
+    replay_unfused(args.steps, start=args.warmup)
+    u1.record()
+    torch.cuda.synchronize(dev)
+    unfused_ms = u0.elapsed_time(u1) / args.steps
+    proj_ms = kt[0] / ksteps
+    flops = 2.0 * R * V * D
+    peak, peak_kind = measured_tensor_peak()
+    achieved = flops / (proj_ms / 1e3) / 1e12
+    line = {
+        "metric": METRIC, "value": args.steps / (ms / 1e3),
+        "unit": f"steps/s (one step = {R} hypotheses x {V} words, hidden size {D}, projection fused into the step)",
+        "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 x bf16 -> f32", "data": "synthetic",
+        "config": {"workload": wl.name + "-fused", "B": wl.B, "k": wl.k, "V": V, "D": D, "rows": R, "stream_steps": T,
+                   "l2": f"operands per step: {R * D * 2 >> 20} MiB of hidden states ({T} rotating buffers) and "
+                         f"{V * D * 2 >> 20} MiB of embedding, which is larger than L2",
+                   "parallelism": "single GPU", "completed_sentences": int((flags & 1).sum())},
+        "kernel_ms": {"projection_scan_and_merge": proj_ms, "constraint_logits_and_candidates": kt[1] / ksteps},
+        "unfused_for_comparison": {"ms_per_step": unfused_ms,
+                                   "what": "torch.matmul (library GEMM, bf16 logits written to HBM) followed by dba_step on them"},
+        "roofline": {"bound": "tensor", "kernel": "project_scan", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "flops_per_launch": flops, "traffic": None},
+        "gpu_launches": launches, "clocks": sampler.result(), "cpu_baseline": None,
+        "e2e": None,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse()
     if args.impl == "reference":
         run_reference(args)
+    elif args.fused:
+        run_fused(args)
     else:
         run_ours(args)
 

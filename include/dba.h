@@ -198,7 +198,8 @@ dba_status dba_finalize(dba_handle* h, int32_t* tokens_host, int32_t* len_host, 
 
 /*
  * Optional per-kernel timing for benchmarks.  While enabled, dba_step brackets each of its two kernels
- * (row scan; candidates with the allocation at their end) with CUDA events on the handle's stream.
+ * (row scan; candidates with the allocation at their end) with CUDA events on the handle's stream; dba_step_fused
+ * brackets the projection with its merge, and the rest (constraint-token logits, candidates).
  * dba_timing_read waits for the stream, adds up the elapsed milliseconds of every step recorded since the last
  * read into ms_total[0..1] (ms_total[2] is 0: the allocation has no kernel of its own), stores the number of
  * steps in *steps and clears the record.  At most 4096 steps are
@@ -263,9 +264,9 @@ dba_status dba_row_scan(const void* logits_dev, int32_t logit_dtype, int32_t R, 
  *   hidden_dev [R, D] bf16, rows hidden_stride_elems apart;  embed_dev [V, D] bf16, rows embed_stride_elems apart;
  *   both 16-byte aligned with strides that are multiples of 8 elements; D a multiple of 8.  n_top <= 32.
  *   Other shapes: DBA_ERR_UNSUPPORTED.  scratch_dev must hold dba_project_scan_scratch_bytes (for the current device).
- * Enqueues on `cuda_stream`, does not synchronise.  A failed device-side wait, or a row with more than 64 logits tied
- * at its n_top-th largest value inside one stretch of the vocabulary, is reported as for dba_row_scan: every row's
- * result is replaced by row_lse = NaN and a list of (-inf, -1).
+ * Enqueues on `cuda_stream`, does not synchronise.  A failed device-side wait, or a row in which more than about 32
+ * logits of one stretch of the vocabulary tie (to bf16 precision) at its n_top-th largest value, is reported as for
+ * dba_row_scan: every row's result is replaced by row_lse = NaN and a list of (-inf, -1).
  */
 dba_status dba_project_scan_scratch_bytes(int32_t R, int32_t V, int32_t n_top, size_t* bytes);
 dba_status dba_project_scan(const void* hidden_dev, int64_t hidden_stride_elems, const void* embed_dev,

@@ -155,6 +155,7 @@ ProjPieces carve_pieces(Carver& cv, size_t R, int P) {
     const size_t cap = (size_t)project_list_cap();
     q.ref = cv.take<int32_t>(R * P); q.sum = cv.take<float>(R * P); q.n = cv.take<int32_t>(R * P);
     q.val = cv.take<float>(R * P * cap); q.col = cv.take<int32_t>(R * P * cap);
+    q.row_tau = cv.take<uint32_t>(R);
     return q;
 }
 
@@ -198,6 +199,22 @@ size_t carve(dba_handle* h, void* base, int32_t max_steps) {
 }
 
 inline dba_status cuda_fail(cudaError_t e) { return e == cudaSuccess ? DBA_OK : DBA_ERR_CUDA; }
+
+// The three events of a recorded step (null when timing is off or the record is full).  False: event creation failed.
+bool step_events(dba_handle* h, cudaEvent_t** ev) {
+    *ev = nullptr;
+    if (!h->timing || h->ev_steps >= kTimingCap) return true;
+    if ((int)h->ev.size() < 3 * (h->ev_steps + 1)) {
+        for (int i = 0; i < 3; ++i) {
+            cudaEvent_t x;
+            if (cudaEventCreate(&x) != cudaSuccess) return false;
+            h->ev.push_back(x);
+        }
+    }
+    *ev = &h->ev[3 * h->ev_steps];
+    h->ev_steps += 1;
+    return true;
+}
 
 }  // namespace
 
@@ -280,17 +297,7 @@ dba_status dba_step(dba_handle* h, const void* logits_dev, int64_t row_stride_el
     const Beam& nxt = h->beam[h->cur ^ 1];
     h->launches_tmp = 0;
     cudaEvent_t* ev = nullptr;
-    if (h->timing && h->ev_steps < kTimingCap) {
-        if ((int)h->ev.size() < 3 * (h->ev_steps + 1)) {
-            for (int i = 0; i < 3; ++i) {
-                cudaEvent_t x;
-                if (cudaEventCreate(&x) != cudaSuccess) return DBA_ERR_CUDA;
-                h->ev.push_back(x);
-            }
-        }
-        ev = &h->ev[3 * h->ev_steps];
-        h->ev_steps += 1;
-    }
+    if (!step_events(h, &ev)) return DBA_ERR_CUDA;
     cudaError_t e = cudaSuccess;
     bool partial = false;
     if (ev) e = cudaEventRecord(ev[0], h->stream);
@@ -324,11 +331,15 @@ dba_status dba_step_fused(dba_handle* h, const void* hidden_dev, int64_t hidden_
     const Beam& cur = h->beam[h->cur];
     const Beam& nxt = h->beam[h->cur ^ 1];
     h->launches_tmp = 0;
+    cudaEvent_t* ev = nullptr;
+    if (!step_events(h, &ev)) return DBA_ERR_CUDA;
     // the list of open rows is not used by this path (every row is projected), but its count is kept in step
     cudaError_t e = cudaMemsetAsync(h->open_count + ((h->t + 1) & 1), 0, sizeof(int32_t), h->stream);
+    if (ev && e == cudaSuccess) e = cudaEventRecord(ev[0], h->stream);
     if (e == cudaSuccess)
         e = launch_project_scan(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, h->d.R, h->d.V, D, h->d.K1,
                                 h->proj, h->proj_stride, h->top, h->status, h->sm_count, h->stream, &h->launches_tmp);
+    if (ev && e == cudaSuccess) e = cudaEventRecord(ev[1], h->stream);
     if (e == cudaSuccess)
         e = launch_constraint_logits(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, D, h->d, h->cons,
                                      h->s2_logit, h->stream, &h->launches_tmp);
@@ -336,6 +347,7 @@ dba_status dba_step_fused(dba_handle* h, const void* hidden_dev, int64_t hidden_
         e = launch_candidates(nullptr, 0, h->d, h->cons, cur, nxt, h->top, ScanScratch{}, nullptr, h->s2_logit, out,
                               h->hist_bp + (size_t)h->t * h->d.R, h->hist_tok + (size_t)h->t * h->d.R, h->status,
                               h->open_list, h->open_count + ((h->t + 1) & 1), h->cand, h->stream, &h->launches_tmp);
+    if (ev && e == cudaSuccess) e = cudaEventRecord(ev[2], h->stream);
     h->launches += h->launches_tmp;
     if (e != cudaSuccess) return DBA_ERR_CUDA;
     h->cur ^= 1;

@@ -79,6 +79,7 @@ struct ProjPieces {
     int32_t* n;        // [R*P] candidates the piece holds
     float* val;        // [R*P*cap]
     int32_t* col;      // [R*P*cap]
+    uint32_t* row_tau; // [R] the bound the row's pieces share while the kernel runs (an ordered integer; zeroed per launch)
 };
 
 // Testing aids of the streaming scan (see dba_test_hook in dba.h).

@@ -9,16 +9,19 @@
 //             operands into a ring of shared-memory stages (128-byte swizzle);
 //   warp 1    allocates tensor memory; one thread issues tcgen05.mma (128 x 256 x 16, bf16 in, fp32 out) into one
 //             of two accumulators in tensor memory and commits the stage back to the loader;
-//   warps 4-7 the epilogue: thread t owns row t of the tile.  It reads its 256 logits from tensor memory, 32 at a
-//             time, and keeps, over all the tiles of its run: the sum of 2^(x log2e - c) against a whole-number
+//   warps 4-7 the epilogue (one warpgroup; the code allows more, each taking a share of the columns): a thread
+//             owns one row of the tile (the four warps reach the four quarters of the rows).  It reads its 256
+//             logits from tensor memory, 32 at a time, and keeps, over all the tiles of its run:
+//             the sum of 2^(x log2e - c) against a whole-number
 //             reference c (raised with an exact rescaling when a logit exceeds it), and the candidates for the row's
 //             K1 largest logits.  Selection: logits at or above a bound tau (-inf at first) go to the thread's list
-//             in shared memory; when some list of the warp has fewer than 32 places left, every thread of the warp
-//             raises its tau to the K1-th largest entry of its list (to 16 bits, by a radix selection over the
-//             list) and drops what fell below, so a list settles at K1 entries plus whatever arrived since.
+//             in shared memory; when some list of the warp has fewer than eight places left (columns are taken
+//             eight at a time), every thread of the warp raises its tau to the K1-th largest entry of its list
+//             (to 16 bits, by a radix selection over the list held in registers) and drops what fell below, so a
+//             list settles at K1 entries plus whatever arrived since.
 // At the end of its part of a row block the thread writes its sum and its list (at least K1 entries, all that reach
-// the final tau) as one piece of the row; project_merge_kernel orders the pieces of a row exactly and writes
-// the row's normaliser and its K1 best entries in the row scan's format.
+// the final tau) as one piece of the row; project_merge_kernel
+// orders the pieces of a row exactly and writes the row's normaliser and its K1 best entries in the row scan's format.
 // Every wait on an mbarrier is bounded: a wait that runs out sets the timeout bit of the status word and the
 // CTA winds down (the tensor memory is freed on every path).
 #include <climits>
@@ -39,9 +42,10 @@ constexpr int kBK = 64;                  // depth of a stage: 64 bf16 = 128 byte
 constexpr int kPStages = 3;
 constexpr int kStageA = kBM * kBK * 2;   // 16 KB
 constexpr int kStageB = kBN * kBK * 2;   // 32 KB
-constexpr int kListCap = 64;             // candidates a thread may hold
-constexpr int kEpiThreads = 128;
-constexpr int kProjThreads = 256;
+constexpr int kListCap = 64;             // candidates a thread may hold (K1 <= 32 of them settled, the rest arrivals)
+constexpr int kEpiHalves = 1;            // epilogue warpgroups: each takes an equal share of every tile's columns
+constexpr int kEpiThreads = 128 * kEpiHalves;
+constexpr int kProjThreads = 128 + kEpiThreads;
 constexpr int kTmemCols = 512;           // two accumulators of 256 columns
 constexpr long long kProjWaitClocks = 4000000000LL;      // about two seconds: a wait this long has failed
 
@@ -63,6 +67,7 @@ struct ProjParams {
     int tiles_m, tiles_n;            // tiles along rows and along the vocabulary
     int pieces;                      // most pieces a row may have (stride of the per-piece arrays)
     ProjPieces out;
+    uint32_t* row_tau;               // [R] zero before the launch: the highest bound any piece of the row has reached so far
     uint32_t* status;
 };
 
@@ -230,10 +235,13 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
         }
     } else if (warp >= 4) {
-        // ------------------------------------------------------------------ epilogue: thread t owns row t of the tile
-        const int et = tid - 128;                          // 0..127
+        // ------------------------------------------------------------------ epilogue: a row and a half of the columns per thread
+        const int et = tid - 128;                          // 0..255: place of this thread's list
+        const int half = (warp - 4) >> 2;                  // which half of the columns
+        const int trow = et & 127;                         // row of the tile = lane of tensor memory
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         float cref = kPNoRef, sum = 0.f, tau = neg_inf();
+        uint32_t tau_key = 0;              // tau as an ordered integer (0: none yet)
         int n_list = 0;
         bool lost = false;                 // a candidate found no room in the list: the piece cannot be trusted
         int cur_m = -1;
@@ -242,29 +250,44 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
         auto compact = [&]() {         // raise tau to the K1-th largest entry of the list (to 16 bits) and drop what is below
             if (n_list < p.K1) return;
+            // the keys come into registers once (empty places as key 0, below every real key); the selection
+            // then runs on registers alone
+            uint32_t key[kListCap];
+#pragma unroll
+            for (int e = 0; e < kListCap; ++e) key[e] = e < n_list ? sm.list_key[e][et] : 0u;
             uint32_t best = 0;         // the largest t, a multiple of 2^16, that at least K1 keys reach
 #pragma unroll 1
             for (uint32_t bit = 0x80000000u; bit >= 0x00010000u; bit >>= 1) {
                 const uint32_t t = best | bit;
                 int cnt = 0;
-                for (int e = 0; e < n_list; ++e) cnt += sm.list_key[e][et] >= t;
+#pragma unroll
+                for (int e = 0; e < kListCap; ++e) cnt += key[e] >= t;
                 if (cnt >= p.K1) best = t;
             }
-            tau = best <= 0x007fffffu ? neg_inf() : unord32(best);
-            int kept = 0;
-            for (int e = 0; e < n_list; ++e) {
-                const uint32_t kx = sm.list_key[e][et];
-                const int c = sm.list_col[e][et];
-                if (kx >= best) { sm.list_key[kept][et] = kx; sm.list_col[kept][et] = c; ++kept; }
+            if (best <= 0x007fffffu) best = 0;
+            // A row's pieces are worked on at the same time by other threads (other CTAs): the K1-th largest entry
+            // of any piece bounds the row's K1-th largest from below, so the pieces share the highest bound found.
+            if (best > tau_key) {
+                tau_key = best;
+                if (cur_m * kBM + et < p.R) atomicMax(p.row_tau + cur_m * kBM + et, best);
             }
+            best = tau_key;
+            tau = tau_key ? unord32(tau_key) : neg_inf();
+            int kept = 0;
+#pragma unroll
+            for (int e = 0; e < kListCap; ++e)
+                if (e < n_list && key[e] >= best) {
+                    const int c = sm.list_col[e][et];          // (kept <= e: nothing unread is overwritten)
+                    sm.list_key[kept][et] = key[e]; sm.list_col[kept][et] = c; ++kept;
+                }
             n_list = kept;
         };
         auto flush = [&](int m, int piece) {      // write this thread's piece of row m * kBM + et
             compact();
-            const int row = m * kBM + et;
+            const int row = m * kBM + trow;
             if (row < p.R) {
                 if (lost) atomicOr(p.status, kStatusOverflow);
-                const int64_t slot = (int64_t)row * p.pieces + piece;
+                const int64_t slot = (int64_t)row * p.pieces + piece * kEpiHalves + half;
                 p.out.ref[slot] = cref != kPNoRef ? __float2int_rn(cref) : INT_MIN;
                 p.out.sum[slot] = sum;
                 p.out.n[slot] = n_list;
@@ -290,15 +313,19 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             if (m != cur_m) {
                 if (cur_m >= 0) flush(cur_m, (int)blockIdx.x - first_cta(cur_m));
                 cur_m = m;
-                cref = kPNoRef; sum = 0.f; tau = neg_inf(); n_list = 0; lost = false;
+                cref = kPNoRef; sum = 0.f; tau = neg_inf(); tau_key = 0; n_list = 0; lost = false;
             }
             const uint32_t acc = tile_no & 1u, acc_use = tile_no >> 1;
+            // what the row's other pieces have found meanwhile (asked for before the wait, used after it)
+            uint32_t seen = 0;
+            if (m * kBM + et < p.R) asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(seen) : "l"(p.row_tau + m * kBM + et));
             if (!__all_sync(kFullMask, pbar_wait(psmem_u32(&sm.acc_full[acc]), acc_use & 1u, abort_flag))) { ok = false; break; }
             tmem_fence_after();
+            if (seen > tau_key) { tau_key = seen; tau = unord32(seen); }
             const int col0 = nn * kBN;
             const bool ragged = col0 + kBN > p.V;           // the vocabulary ends inside this tile
 #pragma unroll 1
-            for (int ch = 0; ch < kBN / 32; ++ch) {
+            for (int ch = half * (kBN / 32 / kEpiHalves); ch < (half + 1) * (kBN / 32 / kEpiHalves); ++ch) {
                 float x[32];
                 tmem_ld32(tmem_base + lane_base + acc * kBN + ch * 32, x);
                 const int cbase = col0 + ch * 32;
@@ -306,16 +333,26 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #pragma unroll
                     for (int c = 0; c < 32; ++c) if (cbase + c >= p.V) x[c] = neg_inf();
                 }
-                float cm = x[0];
+                // candidates, eight columns at a time: most groups hold none, and a group needs at most eight places
+                float cm = neg_inf();
 #pragma unroll
-                for (int c = 1; c < 32; ++c) cm = fmaxf(cm, x[c]);
-                if (cm >= tau && cm != neg_inf()) {
+                for (int g8 = 0; g8 < 4; ++g8) {
+                    float gm = x[g8 * 8];
 #pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        if (x[c] >= tau && x[c] != neg_inf()) {
-                            if (n_list < kListCap) { sm.list_key[n_list][et] = ord32(x[c]); sm.list_col[n_list][et] = cbase + c; ++n_list; }
-                            else lost = true;
+                    for (int c = 1; c < 8; ++c) gm = fmaxf(gm, x[g8 * 8 + c]);
+                    cm = fmaxf(cm, gm);
+                    if (gm >= tau && gm != neg_inf()) {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const float xc = x[g8 * 8 + c];
+                            if (xc >= tau && xc != neg_inf()) {
+                                if (n_list < kListCap) { sm.list_key[n_list][et] = ord32(xc); sm.list_col[n_list][et] = cbase + g8 * 8 + c; ++n_list; }
+                                else lost = true;
+                            }
                         }
+                    }
+                    // room for the next eight columns in every list of the warp, or everybody tidies up now
+                    if (__any_sync(kFullMask, n_list > kListCap - 8)) compact();
                 }
                 // the normaliser
                 const float need = cm * kPLog2e;
@@ -332,8 +369,6 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     s2 += pex2(fmaf(x[c + 2], kPLog2e, -cref)); s3 += pex2(fmaf(x[c + 3], kPLog2e, -cref));
                 }
                 sum += (s0 + s1) + (s2 + s3);
-                // room for the next 32 columns in every list of the warp, or everybody tidies up now
-                if (__any_sync(kFullMask, n_list > kListCap - 32)) compact();
             }
             // the accumulator may be overwritten
             tmem_fence_before();
@@ -366,7 +401,7 @@ __global__ void project_merge_kernel(ProjParams p, int grid_scan, RowTop top) {
         return (int)c;
     };
     const int c0 = owner((long long)m * p.tiles_n), c1 = owner((long long)(m + 1) * p.tiles_n - 1);
-    const int n_pieces = c1 - c0 + 1;
+    const int n_pieces = (c1 - c0 + 1) * kEpiHalves;
     const int64_t base = (int64_t)row * p.pieces;
     // normaliser: pieces in order
     if (lane == 0) {
@@ -407,21 +442,31 @@ __global__ void project_merge_kernel(ProjParams p, int grid_scan, RowTop top) {
     }
 }
 
-// One warp per (row, constraint position of the row's sentence): the inner product, fp32, lanes striding over D.
-__global__ void constraint_logits_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t hs, const __nv_bfloat16* __restrict__ embed,
-                                         int64_t es, int D, int R, int k, const SentCons* __restrict__ cons, float* __restrict__ out) {
-    const int64_t gw = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    const int r = (int)(gw >> 6), j = (int)(gw & 63);
-    if (r >= R) return;
-    const SentCons& sc = cons[r / k];
-    if (j >= sc.C) return;
-    const __nv_bfloat16* h = hidden + (int64_t)r * hs;
-    const __nv_bfloat16* e = embed + (int64_t)sc.ctok[j] * es;
-    float acc = 0.f;
-    for (int i = lane; i < D; i += 32) acc = fmaf(load_logit<__nv_bfloat16>(h + i), load_logit<__nv_bfloat16>(e + i), acc);
-    acc = warp_sum(acc);
-    if (lane == 0) out[(int64_t)r * kMaxC + j] = acc;
+// One CTA per sentence; its warps share out the (row, constraint position) pairs: the inner products
+// <hidden[r], embed[token j]>, fp32, lanes striding over D two entries at a time (the sentence's rows and tokens
+// stay in L1 while its warps go over them).
+constexpr int kGatherWarps = 32;
+__global__ void __launch_bounds__(kGatherWarps * 32)
+constraint_logits_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t hs, const __nv_bfloat16* __restrict__ embed,
+                         int64_t es, int D, int k, const SentCons* __restrict__ cons, float* __restrict__ out) {
+    const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const SentCons& sc = cons[b];
+    const int C = sc.C;
+    for (int item = warp; item < k * C; item += kGatherWarps) {
+        const int h = item / C, j = item - h * C;
+        const int r = b * k + h;
+        const uint32_t* e = reinterpret_cast<const uint32_t*>(embed + (int64_t)sc.ctok[j] * es);
+        const uint32_t* x = reinterpret_cast<const uint32_t*>(hidden + (int64_t)r * hs);
+        float acc = 0.f;
+#pragma unroll 4
+        for (int i = lane; i < D / 2; i += 32) {
+            const uint32_t xw = __ldg(x + i), ew = __ldg(e + i);
+            acc = fmaf(__uint_as_float(xw << 16), __uint_as_float(ew << 16), acc);
+            acc = fmaf(__uint_as_float(xw & 0xffff0000u), __uint_as_float(ew & 0xffff0000u), acc);
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) out[(int64_t)r * kMaxC + j] = acc;
+    }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -458,10 +503,8 @@ bool make_map(CUtensorMap* map, const void* base, int rows, int D, int64_t strid
 
 cudaError_t launch_constraint_logits(const void* hidden, int64_t hidden_stride, const void* embed, int64_t embed_stride,
                                      int D, const Dims& d, const SentCons* cons, float* out, cudaStream_t st, int* launches) {
-    const int64_t warps = (int64_t)d.R * kMaxC;
-    const int per_block = 8;
-    constraint_logits_kernel<<<(unsigned)((warps + per_block - 1) / per_block), per_block * 32, 0, st>>>(
-        (const __nv_bfloat16*)hidden, hidden_stride, (const __nv_bfloat16*)embed, embed_stride, D, d.R, d.k, cons, out);
+    constraint_logits_kernel<<<d.B, kGatherWarps * 32, 0, st>>>(
+        (const __nv_bfloat16*)hidden, hidden_stride, (const __nv_bfloat16*)embed, embed_stride, D, d.k, cons, out);
     ++*launches;
     return cudaGetLastError();
 }
@@ -470,7 +513,7 @@ int project_pieces(int R, int V, int sm_count) {
     const int tiles_m = (R + kBM - 1) / kBM, tiles_n = (V + kBN - 1) / kBN;
     const long long n_tiles = (long long)tiles_m * tiles_n;
     const int grid = (int)(n_tiles < sm_count ? n_tiles : sm_count);
-    return (grid + tiles_m - 1) / tiles_m + 2;
+    return ((grid + tiles_m - 1) / tiles_m + 2) * kEpiHalves;
 }
 
 int project_list_cap() { return kListCap; }
@@ -493,7 +536,9 @@ cudaError_t launch_project_scan(const void* hidden, int64_t hidden_stride, const
     ProjParams p;
     p.R = R; p.V = V; p.D = D; p.K1 = K1;
     p.tiles_m = (R + kBM - 1) / kBM; p.tiles_n = (V + kBN - 1) / kBN;
-    p.pieces = piece_stride; p.out = pieces; p.status = status;
+    p.pieces = piece_stride; p.out = pieces; p.row_tau = pieces.row_tau; p.status = status;
+    cudaError_t e0 = cudaMemsetAsync(pieces.row_tau, 0, sizeof(uint32_t) * (size_t)R, st);
+    if (e0 != cudaSuccess) return e0;
     const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
     const int grid = (int)(n_tiles < sm_count ? n_tiles : sm_count);
     project_scan_kernel<<<grid, kProjThreads, sizeof(ProjSmem) + 1024, st>>>(map_a, map_b, p);

@@ -225,21 +225,32 @@ template <> struct Vec<__nv_bfloat16> {
 // The items of this CTA, in the order all roles agree on.
 // Items are numbered row-major over (position in the list of open rows, segment); this CTA takes every
 // gridDim.x-th one.  The walk needs no division after the constructor.
+// (Only a row's last segment differs from the others in length: what depends on the length alone -- bytes, chunks,
+// the tap of the reports -- is worked out once for the two kinds, and an item picks one.)
 struct ItemIter {
-    int i, seg_, n_rows, S, step_i, step_seg, seg_bytes_full, row_bytes;
-    int bytes_, n_chunks_;        // of the current item
+    int i, seg_, n_rows, S, step_i, step_seg;
+    int bytes_kind[2], chunks_kind[2], tap_kind[2];     // [0]: a full segment, [1]: the row's last segment
+    int bytes_, n_chunks_, tap_;  // of the current item
     uint32_t n_item;
     __device__ ItemIter(const Params& p, int elem_bytes) : S(p.S), n_item(0) {
         n_rows = p.open_count ? *p.open_count : p.R;
         i = blockIdx.x / S; seg_ = blockIdx.x - i * S;
         step_i = gridDim.x / S; step_seg = gridDim.x - step_i * S;
-        seg_bytes_full = p.seg_len * elem_bytes;
-        row_bytes = p.V * elem_bytes;
+        const int seg_bytes_full = p.seg_len * elem_bytes, row_bytes = p.V * elem_bytes;
+        bytes_kind[0] = seg_bytes_full;
+        bytes_kind[1] = row_bytes - (S - 1) * seg_bytes_full;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            chunks_kind[q] = (bytes_kind[q] + kChunkBytes - 1) / kChunkBytes;
+            tap_kind[q] = tap_for(bytes_kind[q], p.K1);
+        }
         load();
     }
     __device__ __forceinline__ void load() {
-        bytes_ = min(seg_bytes_full, row_bytes - seg_ * seg_bytes_full);
-        n_chunks_ = (bytes_ + kChunkBytes - 1) / kChunkBytes;
+        const bool last = seg_ == S - 1;
+        bytes_ = last ? bytes_kind[1] : bytes_kind[0];
+        n_chunks_ = last ? chunks_kind[1] : chunks_kind[0];
+        tap_ = last ? tap_kind[1] : tap_kind[0];
     }
     __device__ bool valid() const { return i < n_rows; }
     __device__ void next() {
@@ -267,12 +278,14 @@ struct ItemIter {
     // values are recorded; G is the largest of 4, 8, 16, 32 that keeps the item at 64 reports or fewer, or, if
     // that is fewer than K1, the smallest that gives K1.
     // tap < 0: no usable bound, every entry is kept.
-    __device__ int report_warps() const {
-        const int nvec = bytes_ >> 4;
+    static __device__ int warps_reporting(int bytes) {
+        const int nvec = bytes >> 4;
         return nvec / kChunkVecs + ((nvec % kChunkVecs) >= 32 ? 1 : 0);
     }
-    __device__ int report_tap(int K1) const {
-        const int warps = report_warps();
+    __device__ int report_warps() const { return warps_reporting(bytes_); }
+    __device__ int report_tap(int) const { return tap_; }
+    static __device__ int tap_for(int bytes, int K1) {
+        const int warps = warps_reporting(bytes);
         if (warps == 0) return -1;
         // as many reports as the selector's fast path takes (64): the more reports, the tighter the bound
         for (int tap = 0; tap <= 3; ++tap)             // G = 32, 16, 8, 4
@@ -333,10 +346,11 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
             ItemIter it(p, (int)sizeof(T)), ahead = it;
             bool ok = true;
             // the row numbers come from a list in global memory: they are asked for kSlots items ahead, so that
-            // no copy waits for one (the first kSlots loads overlap one another)
+            // no copy waits for one (the first kSlots loads overlap one another, and the load of the list's length:
+            // a place beyond the length is still a place of the list, its value is just not used)
             int rows[kSlots];
 #pragma unroll
-            for (int j = 0; j < kSlots; ++j) { rows[j] = ahead.valid() ? ahead.row(p.open_list) : 0; ahead.next(); }
+            for (int j = 0; j < kSlots; ++j) { rows[j] = ahead.i < p.R ? ahead.row(p.open_list) : 0; ahead.next(); }
 #pragma unroll 1
             while (ok && it.valid()) {
 #pragma unroll
@@ -344,7 +358,7 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
                     if (!it.valid()) break;
                     const uint32_t slot = j;
                     const int row = rows[j];
-                    rows[j] = ahead.valid() ? ahead.row(p.open_list) : 0;
+                    rows[j] = ahead.i < p.R ? ahead.row(p.open_list) : 0;
                     ahead.next();
                     if (!mbar_try_wait(smem_u32(&sm.loaded[slot]), it.slot_phase() ^ 1u) &&
                         !mbar_wait(smem_u32(&sm.loaded[slot]), it.slot_phase() ^ 1u, abort_flag)) { ok = false; break; }

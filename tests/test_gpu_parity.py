@@ -170,10 +170,10 @@ def test_fused_step_follows_the_oracle_on_the_projected_logits(dba):
     e = rng.normal(0, 1, (V, D)).astype(np.float32) / np.float32(np.sqrt(D))
     e[:, 0] = mu
     e[:, 1] = 0.0; e[2, 1] = 1.0                     # the end token's logit follows hidden[:, 1]
-    for c in cons:                                   # constraint tokens are likely words
+    for c in cons:                                   # constraint tokens are among the likeliest words
         for ph in c:
             for w in ph:
-                e[w, 0] = -1.0
+                e[w, 0] = 1.5
     eb = to_bf16_bits(e)
     ed = torch.from_numpy(eb.view(np.int16)).cuda().view(torch.bfloat16)
     st = dba.DbaStepper(B, k, V, steps, constraints=cons, dtype=dba.F32, flags=dba.FLAG_FUSED_PROJECTION)
@@ -183,7 +183,7 @@ def test_fused_step_follows_the_oracle_on_the_projected_logits(dba):
     for t in range(steps):
         h = rng.normal(0, 1, (B * k, D)).astype(np.float32)
         h[:, 0] = 1.0
-        h[:, 1] = -6.0 if t < 8 else 4.0             # the end token becomes likely in the second half
+        h[:, 1] = -6.0 if t < 8 else 12.0            # the end token becomes by far the likeliest in the second half
         hb = to_bf16_bits(h)
         X = O.project(hb, eb)
         orc.step(X)
