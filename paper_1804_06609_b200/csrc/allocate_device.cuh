@@ -38,7 +38,7 @@ struct AllocIn {
 // its open rows to the list the next step's row scan reads (the order of that list varies from run to run; no
 // result depends on it).
 __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, const AllocIn& in, const Beam& nxt,
-                                                  const float* __restrict__ row_lse, const dba_step_out& out,
+                                                  const dba_step_out& out,
                                                   int32_t* __restrict__ hist_bp, int32_t* __restrict__ hist_tok,
                                                   int32_t* __restrict__ open_list, int32_t* __restrict__ open_count) {
     __shared__ int n[kBanks];
@@ -48,6 +48,7 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
     __shared__ float a_score[kMaxK];
     __shared__ int a_flat[kMaxK];
     __shared__ int a_tok[kMaxK];
+    __shared__ int a_h[kMaxK];
     __shared__ float a_val[kMaxK];     // what a hypothesis enters the pruning comparison with
     const int lane = threadIdx.x & 31;
     const int k = d.k, V = d.V;
@@ -139,7 +140,13 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
     if (lane == 0) off[0] = ns_total;   // (kept where the code below reads it)
     __syncwarp();
     const int ns = off[0];
-    for (int i = lane; i < ns; i += 32) { const int id = order[sel[i]]; sel[i] = id; a_score[i] = c_score[id]; a_flat[i] = c_flat[id]; }
+    // the selected cells: score, flat index, and (one division per cell) the row it extends and its token
+    for (int i = lane; i < ns; i += 32) {
+        const int id = order[sel[i]];
+        const int fi = c_flat[id];
+        const int h = fi / V;
+        sel[i] = id; a_score[i] = c_score[id]; a_flat[i] = fi; a_h[i] = h; a_tok[i] = fi - h * V;
+    }
     __syncwarp();
     // Section 4: threshold pruning.  Hypotheses whose value is below (best completed value - threshold) are
     // removed, completed or not, and the ones behind them move up.  The value is the cumulative score; with
@@ -148,10 +155,9 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
     if (d.prune > 0.f) {
         float best = neg_inf();
         for (int i = lane; i < ns; i += 32) {
-            const int fi = a_flat[i];
-            const int h = fi / V, w = fi - h * V;
+            const int h = a_h[i];
             float v = a_score[i];
-            if (w == d.eos_id) {
+            if (a_tok[i] == d.eos_id) {
                 if (d.flags & DBA_FLAG_PRUNE_NORMALISED) {
                     const int len = par_kind[h] == 2 ? par_len[h] : par_len[h] + 1;
                     if (len > 0) v = __fdiv_rn(v, (float)len);
@@ -164,26 +170,38 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
         if (best != neg_inf()) cut = __fsub_rn(best, d.prune);
         __syncwarp();
     }
-    // new beam in decreasing score order, ties by lower flat index (Section 3.1), empty slots last
     const int r0 = b * k;
     const bool pruning = cut != neg_inf();
-    int n_pruned = 0;
-    if (pruning)
-        for (int i0 = 0; i0 < ns; i0 += 32) n_pruned += __popc(__ballot_sync(kFullMask, i0 + lane < ns && a_val[i0 + lane] < cut));
-    for (int i = lane; i < k; i += 32) {
-        if (i < ns && !(pruning && a_val[i] < cut)) {
+    // Who stays, who of those is completed; the places of the open ones in the list the next step's row scan reads
+    // are reserved now (a round trip to memory that the ordering and the writes below cover).
+    int n_live = 0, n_done = 0, n_open = 0, list_base = 0;
+    for (int i0 = 0; i0 < ns; i0 += 32) {
+        const int i = i0 + lane;
+        const bool live = i < ns && !(pruning && a_val[i] < cut);
+        const bool done = live && a_tok[i] == d.eos_id;
+        n_live += __popc(__ballot_sync(kFullMask, live));
+        n_done += __popc(__ballot_sync(kFullMask, done));
+    }
+    n_open = n_live - n_done;
+    if (lane == 0 && n_open) list_base = atomicAdd(open_count, n_open);
+    // new beam in decreasing score order, ties by lower flat index (Section 3.1), empty slots last
+    int open_before = 0;        // open cells handled in earlier rounds of the loop below
+    for (int i0 = 0; i0 < k; i0 += 32) {
+        const int i = i0 + lane;
+        const bool live = i < ns && !(pruning && a_val[i] < cut);
+        int rank = 0, w = 0;
+        if (live) {
             const float si = a_score[i]; const int fi = a_flat[i];
-            int rank = 0;
             for (int j = 0; j < ns; ++j) rank += cell_better(a_score[j], a_flat[j], si, fi) && !(pruning && a_val[j] < cut);
             const int id = sel[i];
             const uint64_t cmask = c_mask[id]; const int cactive = c_active[id];
-            const int h = fi / V, w = fi - h * V;
+            const int h = a_h[i];
+            w = a_tok[i];
             const int r = r0 + rank;
             const int bank = __popcll(cmask);
             const int len = par_kind[h] == 2 ? par_len[h] : par_len[h] + 1;      // a finished hypothesis stays as long as it was
             nxt.score[r] = si; nxt.token[r] = w; nxt.mask[r] = cmask; nxt.active[r] = cactive; nxt.len[r] = len;
             nxt.bank[r] = bank; nxt.backptr[r] = h;
-            a_tok[rank] = w;
             hist_bp[r] = h; hist_tok[r] = w;
             if (out.backptr) out.backptr[r] = h;
             if (out.token) out.token[r] = w;
@@ -192,8 +210,14 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
             if (out.met_mask) out.met_mask[r] = cmask;
             if (out.active) out.active[r] = cactive;
         }
+        // rows the next step has to scan: live slots that have not generated the end token
+        const bool open = live && w != d.eos_id;
+        const unsigned bal = __ballot_sync(kFullMask, open);
+        const int base = __shfl_sync(kFullMask, list_base, 0);
+        if (open) open_list[base + open_before + __popc(bal & ((1u << lane) - 1u))] = r0 + rank;
+        open_before += __popc(bal);
     }
-    for (int i = ns - n_pruned + lane; i < k; i += 32) {
+    for (int i = n_live + lane; i < k; i += 32) {
         const int r = r0 + i;
         nxt.score[r] = neg_inf(); nxt.token[r] = d.pad_id; nxt.mask[r] = 0; nxt.active[r] = -1; nxt.len[r] = 0;
         nxt.bank[r] = -1; nxt.backptr[r] = 0;
@@ -204,23 +228,6 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
         if (out.bank) out.bank[r] = -1;
         if (out.met_mask) out.met_mask[r] = 0;
         if (out.active) out.active[r] = -1;
-    }
-    if (out.row_lse)
-        for (int i = lane; i < k; i += 32) out.row_lse[r0 + i] = row_lse[r0 + i];
-    // rows the next step has to scan: live slots that have not generated the end token
-    __syncwarp();
-    int n_live = 0, n_done = 0;
-    for (int i0 = 0; i0 < k; i0 += 32) {
-        const int i = i0 + lane;
-        const bool live = i < ns - n_pruned;
-        const bool open = live && a_tok[i] != d.eos_id;
-        n_live += __popc(__ballot_sync(kFullMask, live));
-        n_done += __popc(__ballot_sync(kFullMask, live && !open));
-        const unsigned bal = __ballot_sync(kFullMask, open);
-        int base = 0;
-        if (lane == 0 && bal) base = atomicAdd(open_count, __popc(bal));
-        base = __shfl_sync(kFullMask, base, 0);
-        if (open) open_list[base + __popc(bal & ((1u << lane) - 1u))] = r0 + i;
     }
     // Section 4's stopping rule (everything on the beam completed) and Section 6.4's early stopping (something is)
     if (out.stop && lane == 0)

@@ -14,20 +14,12 @@ namespace {
 
 constexpr int kCandMaxThreads = 1024;      // the host picks 1024, 512 or 256 threads: the most whose scratch fits
 
-struct SortEnt {
-    uint64_t hi;   // bank << 32 | (~ordered score): ascending = bank ascending, score descending
-    uint32_t lo;   // flat index h*V + w, ascending
-    uint32_t id;   // position in the unsorted candidate arrays
-};
-
 struct Layout {   // byte offsets into dynamic shared memory
     int cons, parent, lse, mask, active, kind, eos_ok, plen, s2_x, rt_score, rt_w, rt_n, rt_ptr, s1_h, s1_i, stage, merged,
         tmp_score, tmp_w, tmp_x, c_score, c_flat, c_mask, c_active, order, bank_cnt, sort, total;
-    int n_sort;
 };
 
 __host__ __device__ inline int align_up(int x, int a) { return (x + a - 1) / a * a; }
-__host__ __device__ inline int next_pow2(int x) { int p = 32; while (p < x) p <<= 1; return p; }
 
 __host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand, int n_warps) {
     Layout L;
@@ -61,8 +53,7 @@ __host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand
     L.order = o;     o += 4 * max_cand;
     L.bank_cnt = o;  o += 4 * (kMaxC + 1);
     o = align_up(o, 16);
-    L.n_sort = next_pow2(max_cand);
-    L.sort = o;      o += (int)sizeof(SortEnt) * L.n_sort;
+    L.sort = o;      o += 12 * max_cand;            // ordering keys (8 bytes) and ids (4 bytes) by grouped place
     L.total = o;
     return L;
 }
@@ -116,7 +107,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     uint64_t* c_mask = reinterpret_cast<uint64_t*>(smem + L.c_mask);
     int* c_active = reinterpret_cast<int*>(smem + L.c_active);
     int* bank_cnt = reinterpret_cast<int*>(smem + L.bank_cnt);
-    SortEnt* ent = reinterpret_cast<SortEnt*>(smem + L.sort);
+    unsigned char* ent = smem + L.sort;
     __shared__ int s_ncand, s_ns1;
 
     const int b = blockIdx.x;
@@ -195,9 +186,9 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     for (int h = warp; h < k; h += n_warps) {
         const int r = r0 + h;
         const int kind = s_kind[h];
-        if (kind == 0) { if (lane == 0) { row_lse[r] = 0.f; s_lse[h] = 0.f; } continue; }
+        if (kind == 0) { if (lane == 0) { row_lse[r] = 0.f; s_lse[h] = 0.f; if (out.row_lse) out.row_lse[r] = 0.f; } continue; }
         if (kind == 2) {                      // finished: repeats the end token at an unchanged score
-            if (lane == 0) { rt_n[h] = 1; rt_score[h * k] = s_parent[h]; rt_w[h * k] = d.eos_id; row_lse[r] = 0.f; s_lse[h] = 0.f; }
+            if (lane == 0) { rt_n[h] = 1; rt_score[h * k] = s_parent[h]; rt_w[h * k] = d.eos_id; row_lse[r] = 0.f; s_lse[h] = 0.f; if (out.row_lse) out.row_lse[r] = 0.f; }
             continue;
         }
         float lse;
@@ -234,7 +225,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
                 const float sum = warp_sum(mg != neg_inf() ? sg * expf(mg - M) : 0.f);
                 lse = M == neg_inf() ? neg_inf() : M + logf(sum);
             }
-            if (lane == 0) row_lse[r] = lse;
+            if (lane == 0) { row_lse[r] = lse; if (out.row_lse) out.row_lse[r] = lse; }
             if (lse_in) lse = lse_given;
             if (lane == 0) s_lse[h] = lse;
             parent = s_parent[h];
@@ -272,6 +263,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         } else {
             // the row's K1 largest raw logits (the finished list) as keys in `merged`, and its normaliser
             lse = row_lse[r];
+            if (lane == 0 && out.row_lse) out.row_lse[r] = lse;
             const float lse_given = lse_in ? lse_in[r] : 0.f;
             const int32_t* gi = top.idx + (int64_t)r * K1;
             const float* gv = top.val + (int64_t)r * K1;
@@ -377,8 +369,32 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     }
     __syncthreads();
 
-    // ---- phase B (source 1): the k best cells of the whole matrix, by a k-round tournament of row heads ----
-    if (warp == 0) {
+    // ---- phase B (source 1): the k best cells of the whole matrix -----------------------------------------------
+    if (warp == 0 && k <= 32) {
+        // Every row's list is in (score desc, token asc) order and at most 32 long: the lists are merged one after
+        // the other, one entry per lane, with the bitonic top-32 merge; the first k of the result are the k best
+        // cells.  Keys: ordered score above, inverted flat index below (larger = better).
+        uint64_t acc = 0;
+        for (int h = 0; h < k; ++h) {
+            const uint64_t key = lane < rt_n[h]
+                ? ((uint64_t)ord32(rt_score[h * k + lane]) << 32) | (uint32_t)(0xffffffffu - (uint32_t)(h * V + rt_w[h * k + lane]))
+                : 0ull;
+            acc = h == 0 ? key : merge_top32(acc, key, lane);
+        }
+        const bool have = lane < k && acc != 0ull;
+        const unsigned sel_mask = __ballot_sync(kFullMask, have);
+        const int flat = (int)(0xffffffffu - (uint32_t)acc);
+        const int h = have ? flat / V : -1 - lane;                       // (lanes without a cell match nobody)
+        // a row's cells are taken in its list's order: the cell's place in its row's list is the number of selected
+        // cells of the same row before it
+        const unsigned same = __match_any_sync(kFullMask, h) & sel_mask;
+        if (have) {
+            s1_h[lane] = h; s1_i[lane] = __popc(same & lt_mask);
+            atomicMax(&rt_ptr[h], __popc(same));
+        }
+        if (lane == 0) s_ns1 = __popc(sel_mask);
+    } else if (warp == 0) {
+        // (beams wider than 32: a k-round tournament of row heads)
         // lane l holds the heads of rows l and l + 32: ordered score key and flat index of the best unused cell
         uint32_t ks[2]; int fl[2], ptr[2] = {0, 0};
 #pragma unroll
@@ -522,66 +538,57 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     if (n > d.max_cand) { if (tid == 0) atomicOr(status, kStatusOverflow); n = d.max_cand; }
 
     // ---- group by bank, order inside each bank (Section 3.1): order (bank asc, score desc, flat asc) ---------
-    int n_sort = 32;
-    while (n_sort < n) n_sort <<= 1;
-    for (int i = tid; i < n_sort; i += n_threads) {
-        SortEnt e;
-        if (i < n) {
-            e.hi = ((uint64_t)__popcll(c_mask[i]) << 32) | (uint32_t)(0xffffffffu - ord32(c_score[i]));
-            e.lo = (uint32_t)c_flat[i]; e.id = (uint32_t)i;
-        } else { e.hi = ~0ull; e.lo = 0xffffffffu; e.id = 0; }
-        ent[i] = e;
+    // Banks first (their sizes are known: a counting sort), then every candidate finds its place inside its bank
+    // by counting the bank's candidates that precede it: the work grows with the size of the banks, not with the
+    // number of candidates, and the result does not depend on the order in which the candidates were appended.
+    __shared__ int bank_off[kMaxC + 1];        // where each bank starts in the grouped order
+    __shared__ int bank_cur[kMaxC + 1];
+    uint64_t* gkey = reinterpret_cast<uint64_t*>(ent);                 // by grouped place: ordering key (smaller = earlier)
+    uint32_t* gid = reinterpret_cast<uint32_t*>(gkey + d.max_cand);    //                   candidate id | bank << 16
+    if (warp == 0) {
+        int run = 0;
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+            const int q = lane + 32 * j;
+            const int c = q <= C ? bank_cnt[q] : 0;
+            int incl = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(kFullMask, incl, o); if (lane >= o) incl += t; }
+            if (q <= C) { bank_off[q] = run + incl - c; bank_cur[q] = 0; }
+            run += __shfl_sync(kFullMask, incl, 31);
+        }
     }
     __syncthreads();
-    if (n <= 160) {
-        // short list: every thread counts how many entries precede its own (keys are distinct) and writes it there
-        if (tid < n) {
-            const SortEnt me = ent[tid];
-            int rank = 0;
+    for (int i = tid; i < n; i += n_threads) {
+        const int bk = __popcll(c_mask[i]);
+        const int at = min(bank_off[bk] + atomicAdd(&bank_cur[bk], 1), d.max_cand - 1);
+        gkey[at] = ((uint64_t)(0xffffffffu - ord32(c_score[i])) << 32) | (uint32_t)c_flat[i];
+        gid[at] = (uint32_t)i | ((uint32_t)bk << 16);
+    }
+    __syncthreads();
+    {
+        // `split` neighbouring lanes share one candidate's count when there are threads to spare
+        int split = 1;
+        while (split < 8 && 2 * split * n <= n_threads) split <<= 1;
+        const int per_pass = n_threads / split;
+        for (int base = 0; base < n; base += per_pass) {
+            const int at = base + tid / split, part = tid & (split - 1);
+            int rank = 0, lo = 0;
+            uint32_t id = 0;
+            if (at < n) {
+                const uint64_t mine = gkey[at];
+                id = gid[at];
+                const int bk = (int)(id >> 16);
+                lo = bank_off[bk];
+                const int nb = min(bank_cnt[bk], n - lo);
+                const int chunk = (nb + split - 1) / split;
+                const int j1 = min(nb, (part + 1) * chunk);
 #pragma unroll 4
-            for (int j = 0; j < n; ++j) {
-                const SortEnt o = ent[j];
-                rank += o.hi < me.hi || (o.hi == me.hi && o.lo < me.lo);
+                for (int j = part * chunk; j < j1; ++j) rank += gkey[lo + j] < mine;
             }
-            s_order[rank] = tid;
+            for (int o = 1; o < split; o <<= 1) rank += __shfl_xor_sync(kFullMask, rank, o);
+            if (at < n && part == 0) s_order[min(lo + rank, d.max_cand - 1)] = (int)(id & 0xffffu);
         }
-    } else if (n_sort <= n_threads) {
-        // medium list: bitonic network with one entry per thread; partners less than a warp apart are reached by
-        // shuffles, the others through shared memory
-        SortEnt me = ent[tid < n_sort ? tid : 0];
-        for (int size = 2; size <= n_sort; size <<= 1) {
-            for (int str = size >> 1; str > 0; str >>= 1) {
-                SortEnt o;
-                if (str >= 32) {
-                    __syncthreads();
-                    if (tid < n_sort) ent[tid] = me;
-                    __syncthreads();
-                    o = ent[(tid ^ str) < n_sort ? (tid ^ str) : 0];
-                } else if (tid < n_sort) {                      // (whole warps: n_sort is a multiple of 32)
-                    o.hi = __shfl_xor_sync(kFullMask, me.hi, str);
-                    o.lo = __shfl_xor_sync(kFullMask, me.lo, str);
-                    o.id = __shfl_xor_sync(kFullMask, me.id, str);
-                } else o = me;
-                const bool mine_first = me.hi < o.hi || (me.hi == o.hi && me.lo < o.lo);
-                const bool want_first = ((tid & str) == 0) == ((tid & size) == 0);     // keep the smaller of the pair?
-                if (mine_first != want_first) me = o;
-            }
-        }
-        if (tid < n) s_order[tid] = (int)me.id;
-    } else {
-        for (int size = 2; size <= n_sort; size <<= 1) {
-            for (int str = size >> 1; str > 0; str >>= 1) {
-                for (int t = tid; t < n_sort / 2; t += n_threads) {
-                    const int pos = 2 * t - (t & (str - 1));
-                    SortEnt a = ent[pos], c = ent[pos + str];
-                    const bool gt = a.hi > c.hi || (a.hi == c.hi && a.lo > c.lo);
-                    const bool up = (pos & size) == 0;
-                    if (gt == up) { ent[pos] = c; ent[pos + str] = a; }
-                }
-                __syncthreads();
-            }
-        }
-        for (int i = tid; i < n; i += n_threads) s_order[i] = (int)ent[i].id;
     }
     // ---- ALLOCATE and the new beam (Section 3.2), by one warp ---------------------------------------------
     __syncthreads();
@@ -589,7 +596,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         AllocIn in;
         in.bank_cnt = bank_cnt; in.order = s_order; in.c_score = c_score; in.c_flat = c_flat; in.c_mask = c_mask;
         in.c_active = c_active; in.par_kind = s_kind; in.par_len = s_plen;
-        allocate_sentence(d, b, C, in, nxt, row_lse, out, hist_bp, hist_tok, open_list, open_count);
+        allocate_sentence(d, b, C, in, nxt, out, hist_bp, hist_tok, open_list, open_count);
     }
 }
 

@@ -42,9 +42,11 @@ constexpr int kBK = 64;                  // depth of a stage: 64 bf16 = 128 byte
 constexpr int kPStages = 3;
 constexpr int kStageA = kBM * kBK * 2;   // 16 KB
 constexpr int kStageB = kBN * kBK * 2;   // 32 KB
-constexpr int kListCap = 64;             // candidates a thread may hold (K1 <= 32 of them settled, the rest arrivals)
-constexpr int kEpiHalves = 1;            // epilogue warpgroups: each takes an equal share of every tile's columns
-constexpr int kEpiThreads = 128 * kEpiHalves;
+constexpr int kListCap = 48;             // candidates a thread may hold (K1 <= 32 of them settled, the rest arrivals)
+constexpr int kEpiGroups = 2;            // epilogue warpgroups: one per accumulator, each taking every other tile
+constexpr int kEpiThreads = 128 * kEpiGroups;
+constexpr int kRefreshSlack = 8;         // arrivals beyond K1 after which a list is tidied at the next tile
+constexpr int kMaxRunTiles = 256;        // tiles a CTA may work through: columns are kept relative to its first one, in 16 bits
 constexpr int kProjThreads = 128 + kEpiThreads;
 constexpr int kTmemCols = 512;           // two accumulators of 256 columns
 constexpr long long kProjWaitClocks = 4000000000LL;      // about two seconds: a wait this long has failed
@@ -53,7 +55,7 @@ struct ProjSmem {
     alignas(1024) unsigned char a[kPStages][kStageA];
     alignas(1024) unsigned char b[kPStages][kStageB];
     uint32_t list_key[kListCap][kEpiThreads];   // entry e of thread t at [e][t] (no bank conflicts): the logit as an ordered integer
-    int32_t list_col[kListCap][kEpiThreads];
+    uint16_t list_col[kListCap][kEpiThreads];  // its column, counted from the first column of the CTA's part of the row block
     uint64_t full[kPStages];         // the stage's operands have landed
     uint64_t empty[kPStages];        // the stage's MMAs are done
     uint64_t acc_full[2];            // the accumulator holds a finished tile
@@ -154,6 +156,7 @@ __device__ __forceinline__ float ppow2i(int d) { return d < -126 ? 0.f : __int_a
 
 constexpr float kPLog2e = 1.44269502162933349609375f;
 constexpr float kPNoRef = -1.0e30f;
+constexpr float kTauNone = -3.402823466e38f;     // no bound yet: every finite logit reaches it, -inf does not
 
 __global__ void __launch_bounds__(kProjThreads, 1)
 project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, ProjParams p) {
@@ -171,7 +174,7 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
     if (tid == 0) {
         for (int s = 0; s < kPStages; ++s) { pbar_init(psmem_u32(&sm.full[s]), 1); pbar_init(psmem_u32(&sm.empty[s]), 1); }
-        for (int a = 0; a < 2; ++a) { pbar_init(psmem_u32(&sm.acc_full[a]), 1); pbar_init(psmem_u32(&sm.acc_empty[a]), kEpiThreads / 32); }
+        for (int a = 0; a < 2; ++a) { pbar_init(psmem_u32(&sm.acc_full[a]), 1); pbar_init(psmem_u32(&sm.acc_empty[a]), 4); }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -235,16 +238,16 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
         }
     } else if (warp >= 4) {
-        // ------------------------------------------------------------------ epilogue: a row and a half of the columns per thread
+        // ------------------------------------------------------------------ epilogue: a row of every other tile per thread
         const int et = tid - 128;                          // 0..255: place of this thread's list
-        const int half = (warp - 4) >> 2;                  // which half of the columns
+        const int grp = (warp - 4) >> 2;                   // takes the tiles in accumulator grp (every other tile of the run)
         const int trow = et & 127;                         // row of the tile = lane of tensor memory
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        float cref = kPNoRef, sum = 0.f, tau = neg_inf();
+        float cref = kPNoRef, sum = 0.f, tau = kTauNone;
         uint32_t tau_key = 0;              // tau as an ordered integer (0: none yet)
         int n_list = 0;
         bool lost = false;                 // a candidate found no room in the list: the piece cannot be trusted
-        int cur_m = -1;
+        int cur_m = -1, col_first = 0;     // row block being worked on, and the first column of this CTA's part of it
         bool ok = true;
         uint32_t tile_no = 0;
 
@@ -265,35 +268,36 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (cnt >= p.K1) best = t;
             }
             if (best <= 0x007fffffu) best = 0;
-            // A row's pieces are worked on at the same time by other threads (other CTAs): the K1-th largest entry
-            // of any piece bounds the row's K1-th largest from below, so the pieces share the highest bound found.
+            // A row's pieces are worked on at the same time by other threads (of this CTA and of others): the K1-th
+            // largest entry of any piece bounds the row's K1-th largest from below, so the pieces share the highest
+            // bound found.
             if (best > tau_key) {
                 tau_key = best;
-                if (cur_m * kBM + et < p.R) atomicMax(p.row_tau + cur_m * kBM + et, best);
+                if (cur_m * kBM + trow < p.R) atomicMax(p.row_tau + cur_m * kBM + trow, best);
             }
             best = tau_key;
-            tau = tau_key ? unord32(tau_key) : neg_inf();
+            tau = tau_key ? unord32(tau_key) : kTauNone;
             int kept = 0;
 #pragma unroll
             for (int e = 0; e < kListCap; ++e)
                 if (e < n_list && key[e] >= best) {
-                    const int c = sm.list_col[e][et];          // (kept <= e: nothing unread is overwritten)
+                    const uint16_t c = sm.list_col[e][et];     // (kept <= e: nothing unread is overwritten)
                     sm.list_key[kept][et] = key[e]; sm.list_col[kept][et] = c; ++kept;
                 }
             n_list = kept;
         };
-        auto flush = [&](int m, int piece) {      // write this thread's piece of row m * kBM + et
+        auto flush = [&](int m, int piece) {      // write this thread's piece of row m * kBM + trow
             compact();
             const int row = m * kBM + trow;
             if (row < p.R) {
                 if (lost) atomicOr(p.status, kStatusOverflow);
-                const int64_t slot = (int64_t)row * p.pieces + piece * kEpiHalves + half;
+                const int64_t slot = (int64_t)row * p.pieces + piece * kEpiGroups + grp;
                 p.out.ref[slot] = cref != kPNoRef ? __float2int_rn(cref) : INT_MIN;
                 p.out.sum[slot] = sum;
                 p.out.n[slot] = n_list;
                 for (int e = 0; e < n_list; ++e) {
                     p.out.val[slot * kListCap + e] = unord32(sm.list_key[e][et]);
-                    p.out.col[slot * kListCap + e] = sm.list_col[e][et];
+                    p.out.col[slot * kListCap + e] = col_first + (int)sm.list_col[e][et];
                 }
             }
         };
@@ -310,22 +314,26 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #pragma unroll 1
         for (int t = t_begin; t < t_end && ok; ++t, ++tile_no) {
             const int m = t / p.tiles_n, nn = t - m * p.tiles_n;
-            if (m != cur_m) {
+            if (m != cur_m) {          // (both groups pass here, whoever gets the row block's first tile)
                 if (cur_m >= 0) flush(cur_m, (int)blockIdx.x - first_cta(cur_m));
-                cur_m = m;
-                cref = kPNoRef; sum = 0.f; tau = neg_inf(); tau_key = 0; n_list = 0; lost = false;
+                cur_m = m; col_first = nn * kBN;
+                cref = kPNoRef; sum = 0.f; tau = kTauNone; tau_key = 0; n_list = 0; lost = false;
             }
-            const uint32_t acc = tile_no & 1u, acc_use = tile_no >> 1;
+            if ((tile_no & 1u) != (uint32_t)grp) continue;
+            const uint32_t acc = (uint32_t)grp, acc_use = tile_no >> 1;
             // what the row's other pieces have found meanwhile (asked for before the wait, used after it)
+            const bool live = m * kBM + trow < p.R;            // (the last row block may reach past the last row)
             uint32_t seen = 0;
-            if (m * kBM + et < p.R) asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(seen) : "l"(p.row_tau + m * kBM + et));
+            if (live) asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(seen) : "l"(p.row_tau + m * kBM + trow));
+            // a list that has grown since its bound was last raised is tidied while the tile is still being computed
+            if (__any_sync(kFullMask, n_list >= p.K1 + kRefreshSlack)) compact();
             if (!__all_sync(kFullMask, pbar_wait(psmem_u32(&sm.acc_full[acc]), acc_use & 1u, abort_flag))) { ok = false; break; }
             tmem_fence_after();
             if (seen > tau_key) { tau_key = seen; tau = unord32(seen); }
             const int col0 = nn * kBN;
             const bool ragged = col0 + kBN > p.V;           // the vocabulary ends inside this tile
 #pragma unroll 1
-            for (int ch = half * (kBN / 32 / kEpiHalves); ch < (half + 1) * (kBN / 32 / kEpiHalves); ++ch) {
+            for (int ch = 0; ch < kBN / 32; ++ch) {
                 float x[32];
                 tmem_ld32(tmem_base + lane_base + acc * kBN + ch * 32, x);
                 const int cbase = col0 + ch * 32;
@@ -333,26 +341,45 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #pragma unroll
                     for (int c = 0; c < 32; ++c) if (cbase + c >= p.V) x[c] = neg_inf();
                 }
-                // candidates, eight columns at a time: most groups hold none, and a group needs at most eight places
                 float cm = neg_inf();
 #pragma unroll
-                for (int g8 = 0; g8 < 4; ++g8) {
-                    float gm = x[g8 * 8];
+                for (int c = 0; c < 32; ++c) cm = fmaxf(cm, x[c]);
+                // candidates: the columns at or above the bound (a finite number, so -inf never is), as a bit mask;
+                // they go to the list eight columns at a time, and a list that is full is tidied (which raises
+                // the bound) before the rest is looked at again
+                if (__any_sync(kFullMask, live && cm >= tau)) {
+                    uint32_t mk = 0;
 #pragma unroll
-                    for (int c = 1; c < 8; ++c) gm = fmaxf(gm, x[g8 * 8 + c]);
-                    cm = fmaxf(cm, gm);
-                    if (gm >= tau && gm != neg_inf()) {
+                    for (int c = 0; c < 32; ++c) mk |= (x[c] >= tau ? 1u : 0u) << c;
+                    if (!live) mk = 0;
+#pragma unroll 1
+                    for (int round = 0; ; ++round) {
+                        uint32_t pending = 0;
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            const float xc = x[g8 * 8 + c];
-                            if (xc >= tau && xc != neg_inf()) {
-                                if (n_list < kListCap) { sm.list_key[n_list][et] = ord32(xc); sm.list_col[n_list][et] = cbase + g8 * 8 + c; ++n_list; }
-                                else lost = true;
+                        for (int g8 = 0; g8 < 4; ++g8) {
+                            uint32_t sub = (mk >> (8 * g8)) & 0xffu;
+                            while (sub) {
+                                if (n_list == kListCap) { pending |= sub << (8 * g8); break; }
+                                const int c = __ffs(sub) - 1;
+                                sub &= sub - 1;
+                                const float a0 = (c & 1) ? x[g8 * 8 + 1] : x[g8 * 8], a1 = (c & 1) ? x[g8 * 8 + 3] : x[g8 * 8 + 2];
+                                const float a2 = (c & 1) ? x[g8 * 8 + 5] : x[g8 * 8 + 4], a3 = (c & 1) ? x[g8 * 8 + 7] : x[g8 * 8 + 6];
+                                const float b0 = (c & 2) ? a1 : a0, b1 = (c & 2) ? a3 : a2;
+                                const float v = (c & 4) ? b1 : b0;
+                                sm.list_key[n_list][et] = ord32(v);
+                                sm.list_col[n_list][et] = (uint16_t)(cbase + g8 * 8 + c - col_first);
+                                ++n_list;
                             }
                         }
+                        // (the loop is left by the whole warp together: the votes inside it name every lane)
+                        if (!__any_sync(kFullMask, pending != 0)) break;
+                        compact();
+                        if (pending != 0 && (n_list == kListCap || round >= 8)) { lost = true; pending = 0; }   // more ties than places
+                        mk = 0;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) mk |= (x[c] >= tau ? 1u : 0u) << c;
+                        mk &= pending;
                     }
-                    // room for the next eight columns in every list of the warp, or everybody tidies up now
-                    if (__any_sync(kFullMask, n_list > kListCap - 8)) compact();
                 }
                 // the normaliser
                 const float need = cm * kPLog2e;
@@ -385,11 +412,19 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     if (tid == 0 && sm.abort_flag) atomicOr(p.status, kStatusTimeout);
 }
 
-// Orders the pieces of every row exactly: one warp per row gathers the candidates of the row's pieces, ranks them
-// (value descending, lower index first) and writes the K1 best and the row's normaliser.
-__global__ void project_merge_kernel(ProjParams p, int grid_scan, RowTop top) {
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
+// Orders the pieces of every row exactly: one warp per row adds up the pieces' sums (in the order of the pieces),
+// gathers their candidates into shared memory, finds the value of the K1-th largest a byte at a time (a histogram
+// of the next byte over the entries that share the bytes found so far) and ranks the entries that reach it
+// (value descending, lower column first).  Global memory is read in batches of independent loads: a row costs a
+// few round trips to L2, not one per piece.
+constexpr int kMergeWarps = 4;
+constexpr int kMergeKeys = 1024;         // entries of a row that fit in shared memory (more: they are read in place)
+constexpr int kMergeBuf = 128;           // entries at or above the K1-th largest value that are ranked the short way
+__global__ void __launch_bounds__(kMergeWarps * 32) project_merge_kernel(ProjParams p, int grid_scan, RowTop top) {
+    __shared__ uint64_t s_key[kMergeWarps][kMergeKeys];
+    __shared__ uint32_t s_hist[kMergeWarps][256];
+    const int row = blockIdx.x * kMergeWarps + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     if (row >= p.R) return;
     const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
     const int m = row / kBM;
@@ -401,16 +436,34 @@ __global__ void project_merge_kernel(ProjParams p, int grid_scan, RowTop top) {
         return (int)c;
     };
     const int c0 = owner((long long)m * p.tiles_n), c1 = owner((long long)(m + 1) * p.tiles_n - 1);
-    const int n_pieces = (c1 - c0 + 1) * kEpiHalves;
+    const int n_pieces = (c1 - c0 + 1) * kEpiGroups;
     const int64_t base = (int64_t)row * p.pieces;
-    // normaliser: pieces in order
+    const unsigned lt_mask = (1u << lane) - 1u;
+    uint64_t* keys = s_key[wib];
+    uint32_t* hist = s_hist[wib];
+
+    // ---- normaliser: highest reference first, then the sums rescaled to it, added in the order of the pieces
+    int C = INT_MIN;
+    for (int g0 = 0; g0 < n_pieces; g0 += 32) {
+        const int g = g0 + lane;
+        C = max(C, g < n_pieces ? p.out.ref[base + g] : INT_MIN);
+    }
+    C = __reduce_max_sync(kFullMask, C);
+    float total = 0.f;
+    int total_n = 0, n_first = 0;          // n_first: lane g holds the length of piece g (the first 32 pieces)
+    for (int g0 = 0; g0 < n_pieces; g0 += 32) {
+        const int g = g0 + lane;
+        float term = 0.f; int ng = 0;
+        if (g < n_pieces) {
+            const int ref = p.out.ref[base + g];
+            if (ref != INT_MIN) term = p.out.sum[base + g] * ppow2i(ref - C);
+            ng = p.out.n[base + g];
+        }
+        for (int j = 0; j < min(32, n_pieces - g0); ++j) total += __shfl_sync(kFullMask, term, j);
+        total_n += __reduce_add_sync(kFullMask, ng);
+        if (g0 == 0) n_first = ng;
+    }
     if (lane == 0) {
-        int C = INT_MIN;
-        for (int g = 0; g < n_pieces; ++g) C = max(C, p.out.ref[base + g]);
-        float total = 0.f;
-        if (C != INT_MIN)
-            for (int g = 0; g < n_pieces; ++g)
-                if (p.out.ref[base + g] != INT_MIN) total += p.out.sum[base + g] * ppow2i(p.out.ref[base + g] - C);
         float lse = neg_inf();
         if (C != INT_MIN && total > 0.f) {
             constexpr float kLn2Hi = 0.693147182464599609375f, kLn2Lo = -1.904654299957767e-9f;
@@ -419,11 +472,114 @@ __global__ void project_merge_kernel(ProjParams p, int grid_scan, RowTop top) {
         }
         top.lse[row] = lse;
     }
-    // candidates: entry e of piece g; rank by counting the better ones
+
+    // ---- candidates
     float* tv = top.val + (int64_t)row * p.K1;
     int32_t* ti = top.idx + (int64_t)row * p.K1;
-    int total_n = 0;
-    for (int g = 0; g < n_pieces; ++g) total_n += p.out.n[base + g];
+    const bool in_smem = total_n <= kMergeKeys;
+    if (in_smem) {            // all entries to shared memory, as keys (value above, inverted column below)
+        static_assert(kListCap <= 64, "a piece is read in two rounds of 32");
+        int at = 0;
+#pragma unroll 4
+        for (int g = 0; g < n_pieces; ++g) {
+            const int ng = g < 32 ? __shfl_sync(kFullMask, n_first, g) : p.out.n[base + g];
+            const int64_t pb = (base + g) * kListCap;
+            const bool h0 = lane < ng, h1 = lane + 32 < ng;
+            float v0 = 0.f, v1 = 0.f; int w0 = 0, w1 = 0;
+            if (h0) { v0 = p.out.val[pb + lane]; w0 = p.out.col[pb + lane]; }
+            if (h1) { v1 = p.out.val[pb + lane + 32]; w1 = p.out.col[pb + lane + 32]; }
+            if (h0) keys[at + lane] = row_key(v0, w0);
+            if (h1) keys[at + lane + 32] = row_key(v1, w1);
+            at += ng;
+        }
+        __syncwarp();
+    }
+    // visits the value (as an ordered integer) of every entry of the row
+    auto for_each_value = [&](auto&& f) {
+        if (in_smem) {
+            for (int i = lane; i < total_n; i += 32) f((uint32_t)(keys[i] >> 32));
+        } else {
+            for (int g = 0; g < n_pieces; ++g) {
+                const int ng = p.out.n[base + g];
+                for (int e = lane; e < ng; e += 32) f(ord32(p.out.val[(base + g) * kListCap + e]));
+            }
+        }
+    };
+    uint32_t thr = 0;                       // ordered-integer value of the K1-th largest entry (0: there are no more than K1)
+    if (total_n > p.K1) {
+        uint32_t prefix = 0, prefix_mask = 0;
+        int need = p.K1;                    // the entry looked for is the need-th largest of those that share the prefix
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            for (int i = lane; i < 256; i += 32) hist[i] = 0;
+            __syncwarp();
+            for_each_value([&](uint32_t k32) {
+                if ((k32 & prefix_mask) == prefix) atomicAdd(&hist[(k32 >> shift) & 255u], 1u);
+            });
+            __syncwarp();
+            // lane l holds bytes 8l .. 8l+7; the byte wanted is the highest one with (entries above it) < need
+            uint32_t bins[8], mine = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { bins[j] = hist[lane * 8 + j]; mine += bins[j]; }
+            uint32_t above = mine;          // entries in this lane's bytes and all higher ones
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t up = __shfl_down_sync(kFullMask, above, o);
+                if (lane + o < 32) above += up;
+            }
+            above -= mine;                  // entries in higher lanes' bytes only
+            const bool here = above < (uint32_t)need && above + mine >= (uint32_t)need;
+            int digit = 0; uint32_t over = 0;
+            if (here) {
+                uint32_t acc = above;
+                bool found = false;
+#pragma unroll
+                for (int j = 7; j >= 0; --j) {
+                    if (!found && acc + bins[j] >= (uint32_t)need) { digit = lane * 8 + j; over = acc; found = true; }
+                    acc += bins[j];
+                }
+            }
+            const int src = __ffs(__ballot_sync(kFullMask, here)) - 1;      // exactly one lane
+            digit = __shfl_sync(kFullMask, digit, src); over = __shfl_sync(kFullMask, over, src);
+            need -= (int)over;
+            prefix |= (uint32_t)digit << shift; prefix_mask |= 255u << shift;
+            __syncwarp();
+        }
+        thr = prefix;
+    }
+    // the entries that reach the value, to the front of a short list
+    uint64_t* buf = reinterpret_cast<uint64_t*>(hist);         // (the histogram is done with: 256 words = 128 keys)
+    static_assert(kMergeBuf * 2 <= 256, "the short list lives where the histogram was");
+    int cnt = 0;
+    auto take = [&](bool valid, uint64_t key) {
+        const bool hit = valid && (uint32_t)(key >> 32) >= thr;
+        const unsigned bal = __ballot_sync(kFullMask, hit);
+        const int pos = cnt + __popc(bal & lt_mask);
+        if (hit && pos < kMergeBuf) buf[pos] = key;
+        cnt += __popc(bal);
+    };
+    if (in_smem) {
+        for (int i0 = 0; i0 < total_n; i0 += 32) take(i0 + lane < total_n, i0 + lane < total_n ? keys[i0 + lane] : 0ull);
+    } else {
+        for (int g = 0; g < n_pieces; ++g) {
+            const int ng = p.out.n[base + g];
+            for (int e0 = 0; e0 < ng; e0 += 32) {
+                const int e = e0 + lane;
+                take(e < ng, e < ng ? row_key(p.out.val[(base + g) * kListCap + e], p.out.col[(base + g) * kListCap + e]) : 0ull);
+            }
+        }
+    }
+    __syncwarp();
+    if (cnt <= kMergeBuf) {
+        for (int e = cnt + lane; e < p.K1; e += 32) { tv[e] = neg_inf(); ti[e] = -1; }
+        for (int i = lane; i < cnt; i += 32) {
+            const uint64_t key = buf[i];
+            int rank = 0;
+            for (int j = 0; j < cnt; ++j) rank += buf[j] > key;
+            if (rank < p.K1) { tv[rank] = row_key_val(key); ti[rank] = (int32_t)(0xffffffffu - (uint32_t)key); }
+        }
+        return;
+    }
+    // (more entries tied with the K1-th largest than the short way holds: every entry is ranked among all of them)
     for (int e = total_n + lane; e < p.K1; e += 32) { tv[e] = neg_inf(); ti[e] = -1; }
     for (int g = 0; g < n_pieces; ++g) {
         const int ng = p.out.n[base + g];
@@ -509,11 +665,17 @@ cudaError_t launch_constraint_logits(const void* hidden, int64_t hidden_stride, 
     return cudaGetLastError();
 }
 
+// CTAs of the scan: one per SM, more when a CTA would otherwise get more than kMaxRunTiles tiles
+static int project_grid(long long n_tiles, int sm_count) {
+    const long long by_run = (n_tiles + kMaxRunTiles - 1) / kMaxRunTiles;
+    const long long g = n_tiles < sm_count ? n_tiles : sm_count;
+    return (int)(g > by_run ? g : by_run);
+}
+
 int project_pieces(int R, int V, int sm_count) {
     const int tiles_m = (R + kBM - 1) / kBM, tiles_n = (V + kBN - 1) / kBN;
-    const long long n_tiles = (long long)tiles_m * tiles_n;
-    const int grid = (int)(n_tiles < sm_count ? n_tiles : sm_count);
-    return ((grid + tiles_m - 1) / tiles_m + 2) * kEpiHalves;
+    const int grid = project_grid((long long)tiles_m * tiles_n, sm_count);
+    return ((grid + tiles_m - 1) / tiles_m + 2) * kEpiGroups;
 }
 
 int project_list_cap() { return kListCap; }
@@ -540,13 +702,12 @@ cudaError_t launch_project_scan(const void* hidden, int64_t hidden_stride, const
     cudaError_t e0 = cudaMemsetAsync(pieces.row_tau, 0, sizeof(uint32_t) * (size_t)R, st);
     if (e0 != cudaSuccess) return e0;
     const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
-    const int grid = (int)(n_tiles < sm_count ? n_tiles : sm_count);
+    const int grid = project_grid(n_tiles, sm_count);
     project_scan_kernel<<<grid, kProjThreads, sizeof(ProjSmem) + 1024, st>>>(map_a, map_b, p);
     ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const int warps = 8;
-    project_merge_kernel<<<(R + warps - 1) / warps, warps * 32, 0, st>>>(p, grid, top);
+    project_merge_kernel<<<(R + kMergeWarps - 1) / kMergeWarps, kMergeWarps * 32, 0, st>>>(p, grid, top);
     ++*launches;
     return cudaGetLastError();
 }
