@@ -264,9 +264,11 @@ dba_status dba_row_scan(const void* logits_dev, int32_t logit_dtype, int32_t R, 
  *   hidden_dev [R, D] bf16, rows hidden_stride_elems apart;  embed_dev [V, D] bf16, rows embed_stride_elems apart;
  *   both 16-byte aligned with strides that are multiples of 8 elements; D a multiple of 8.  n_top <= 32.
  *   Other shapes: DBA_ERR_UNSUPPORTED.  scratch_dev must hold dba_project_scan_scratch_bytes (for the current device).
- * Enqueues on `cuda_stream`, does not synchronise.  A failed device-side wait, or a row in which more than about 32
- * logits of one stretch of the vocabulary tie (to bf16 precision) at its n_top-th largest value, is reported as for
- * dba_row_scan: every row's result is replaced by row_lse = NaN and a list of (-inf, -1).
+ * Enqueues on `cuda_stream`, does not synchronise.  A failed device-side wait, or a row of which 48 or more
+ * logits within one stretch of the vocabulary (the part one thread works through: every other 256-word tile of
+ * a run of up to 256 tiles) agree with its n_top-th largest value in sign, exponent and the leading 7 bits of
+ * the mantissa, is reported as for dba_row_scan: every row's result is replaced by row_lse = NaN and a list of
+ * (-inf, -1).
  */
 dba_status dba_project_scan_scratch_bytes(int32_t R, int32_t V, int32_t n_top, size_t* bytes);
 dba_status dba_project_scan(const void* hidden_dev, int64_t hidden_stride_elems, const void* embed_dev,

@@ -14,6 +14,7 @@ struct dba_handle {
     cudaStream_t stream;
     int device;
     int sm_count;
+    int proj_pairs;                // only with DBA_FLAG_FUSED_PROJECTION: pairs of CTAs the device runs at once
     // carved from the caller's workspace
     SentCons* cons;
     Beam beam[2];
@@ -262,7 +263,7 @@ dba_status dba_init(const dba_config* cfg, void* workspace_dev, size_t workspace
     e = configure_candidates(h->d, &h->cand, &fits);
     if (e == cudaSuccess && !fits) { delete h; return DBA_ERR_UNSUPPORTED; }
     if (e == cudaSuccess) e = configure_row_scan_tma();
-    if (e == cudaSuccess && (cfg->flags & DBA_FLAG_FUSED_PROJECTION)) e = configure_project_scan();
+    if (e == cudaSuccess && (cfg->flags & DBA_FLAG_FUSED_PROJECTION)) e = configure_project_scan(&h->proj_pairs);
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(h->cons, cons.data(), sizeof(SentCons) * cons.size(), cudaMemcpyHostToDevice, h->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(h->status, 0, 256, h->stream);
@@ -338,7 +339,7 @@ dba_status dba_step_fused(dba_handle* h, const void* hidden_dev, int64_t hidden_
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[0], h->stream);
     if (e == cudaSuccess)
         e = launch_project_scan(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, h->d.R, h->d.V, D, h->d.K1,
-                                h->proj, h->proj_stride, h->top, h->status, h->sm_count, h->stream, &h->launches_tmp);
+                                h->proj, h->proj_stride, h->top, h->status, h->proj_pairs, h->stream, &h->launches_tmp);
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[1], h->stream);
     if (e == cudaSuccess)
         e = launch_constraint_logits(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, D, h->d, h->cons,
@@ -555,10 +556,11 @@ dba_status dba_project_scan(const void* hidden_dev, int64_t hidden_stride_elems,
     int launches = 0;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     e = cudaMemsetAsync(status, 0, 256, stream);
-    if (e == cudaSuccess) e = configure_project_scan();
+    int max_pairs = 0;
+    if (e == cudaSuccess) e = configure_project_scan(&max_pairs);
     if (e == cudaSuccess)
         e = launch_project_scan(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, R, V, D, n_top, pieces, stride,
-                                top, status, sms, stream, &launches);
+                                top, status, max_pairs, stream, &launches);
     if (e == cudaSuccess) e = launch_scan_check(status, R, n_top, top, stream);
     return cuda_fail(e);
 }

@@ -137,10 +137,10 @@ int max_segments(int V, int dtype);
 int project_pieces(int R, int V, int sm_count);       // pieces a row may have: the stride of ProjPieces
 int project_list_cap();
 bool project_scan_usable(const void* hidden, int64_t hidden_stride, const void* embed, int64_t embed_stride, int D, int K1);
-cudaError_t configure_project_scan();
+cudaError_t configure_project_scan(int* max_pairs);      // *max_pairs: pairs of CTAs the device runs at once
 cudaError_t launch_project_scan(const void* hidden, int64_t hidden_stride, const void* embed, int64_t embed_stride,
                                 int R, int V, int D, int K1, const ProjPieces& pieces, int piece_stride,
-                                const RowTop& top, uint32_t* status, int sm_count, cudaStream_t st, int* launches);
+                                const RowTop& top, uint32_t* status, int max_pairs, cudaStream_t st, int* launches);
 // logits of every sentence's constraint tokens for its rows: out[r * 64 + j] = <hidden[r], embed[token j of the
 // sentence of row r]> (fp32), for the fused step, which has no logit matrix to look them up in
 cudaError_t launch_constraint_logits(const void* hidden, int64_t hidden_stride, const void* embed, int64_t embed_stride,

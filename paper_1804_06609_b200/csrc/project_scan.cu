@@ -2,28 +2,35 @@
 // that Algorithm 2 reads): logits[r, w] = <hidden[r, :], embed[w, :]> are computed on the tensor cores and
 // consumed where they appear, so the R x V matrix never exists in HBM.
 //
-// One persistent CTA per SM.  The tiles (128 rows of hidden states x 256 words) are numbered row block by row
-// block and dealt out in equal contiguous runs, so a CTA works through part of one row block's vocabulary (and
-// possibly the start of the next row block's).  Roles, talking through mbarriers only:
-//   warp 0    one thread issues the TMA loads (cp.async.bulk.tensor, no multicast) of the 64-deep slices of both
-//             operands into a ring of shared-memory stages (128-byte swizzle);
-//   warp 1    allocates tensor memory; one thread issues tcgen05.mma (128 x 256 x 16, bf16 in, fp32 out) into one
-//             of two accumulators in tensor memory and commits the stage back to the loader;
-//   warps 4-7 the epilogue (one warpgroup; the code allows more, each taking a share of the columns): a thread
-//             owns one row of the tile (the four warps reach the four quarters of the rows).  It reads its 256
-//             logits from tensor memory, 32 at a time, and keeps, over all the tiles of its run:
+// Persistent CTAs in pairs (a cluster of two, one CTA per SM).  A pair works on tiles of 256 rows of hidden states
+// x 256 words: each CTA holds its 128 rows of the hidden states and its 128 words of the embedding slice in shared
+// memory, and one tcgen05.mma of the pair (cta_group::2, issued by the pair's first CTA) multiplies the 256 x 256
+// tile, each CTA receiving the accumulator of its own 128 rows in its tensor memory.  That halves what each SM
+// has to fetch of the embedding, which is what bounds a single CTA on a 128 x 256 tile.  The tiles are numbered row
+// block by row block and dealt out to the pairs in equal contiguous runs, so a pair works through part of one row
+// block's vocabulary (and possibly the start of the next row block's).  Roles in each CTA, talking through mbarriers:
+//   warp 0    one thread issues the TMA loads (cp.async.bulk.tensor, cta_group::2, no multicast) of the 64-deep
+//             slices of this CTA's halves of both operands into a ring of shared-memory stages (128-byte swizzle);
+//             the bytes of both CTAs are counted on the first CTA's barrier;
+//   warp 1    allocates tensor memory (both CTAs); in the first CTA one thread issues the pair's tcgen05.mma
+//             (256 x 256 x 16, bf16 in, fp32 out) into one of two accumulators and commits the stage back to both
+//             loaders, and the finished accumulator to both epilogues;
+//   warps 4-11 the epilogue: two warpgroups, one per accumulator, each taking every other tile of the run.  A thread
+//             owns one row of the tile (the four warps of a group reach the four quarters of the CTA's rows).  It
+//             reads its 256 logits from tensor memory, 32 at a time, and keeps, over all its tiles of the run:
 //             the sum of 2^(x log2e - c) against a whole-number
 //             reference c (raised with an exact rescaling when a logit exceeds it), and the candidates for the row's
-//             K1 largest logits.  Selection: logits at or above a bound tau (-inf at first) go to the thread's list
-//             in shared memory; when some list of the warp has fewer than eight places left (columns are taken
-//             eight at a time), every thread of the warp raises its tau to the K1-th largest entry of its list
-//             (to 16 bits, by a radix selection over the list held in registers) and drops what fell below, so a
-//             list settles at K1 entries plus whatever arrived since.
+//             K1 largest logits.  Selection: logits at or above a bound tau (none at first) go to the thread's list
+//             in shared memory (found as a bit mask over the 32 columns); when a list is full, every thread of the
+//             warp raises its tau to the K1-th largest entry of its list (to 16 bits, by a radix selection over the
+//             list held in registers) and drops what fell below, so a list settles at K1 entries plus whatever
+//             arrived since.  The bound is shared among all threads working on the same row (an atomic maximum in
+//             global memory, read again before every tile).
 // At the end of its part of a row block the thread writes its sum and its list (at least K1 entries, all that reach
 // the final tau) as one piece of the row; project_merge_kernel
 // orders the pieces of a row exactly and writes the row's normaliser and its K1 best entries in the row scan's format.
 // Every wait on an mbarrier is bounded: a wait that runs out sets the timeout bit of the status word and the
-// CTA winds down (the tensor memory is freed on every path).
+// CTA winds down (the tensor memory is freed on every path); the two CTAs of a pair leave together.
 #include <climits>
 
 #include <cuda.h>
@@ -36,12 +43,14 @@ namespace dba {
 
 namespace {
 
-constexpr int kBM = 128;                 // rows of hidden states per tile (= lanes of tensor memory)
+constexpr int kBM = 128;                 // rows of hidden states per CTA and tile (= lanes of tensor memory)
+constexpr int kPairM = 2 * kBM;          // rows of a pair's tile
 constexpr int kBN = 256;                 // words per tile (= columns of one accumulator)
+constexpr int kHalfN = kBN / 2;          // words of the tile whose embedding rows this CTA holds
 constexpr int kBK = 64;                  // depth of a stage: 64 bf16 = 128 bytes, one swizzle row
-constexpr int kPStages = 3;
+constexpr int kPStages = 4;
 constexpr int kStageA = kBM * kBK * 2;   // 16 KB
-constexpr int kStageB = kBN * kBK * 2;   // 32 KB
+constexpr int kStageB = kHalfN * kBK * 2; // 16 KB
 constexpr int kListCap = 48;             // candidates a thread may hold (K1 <= 32 of them settled, the rest arrivals)
 constexpr int kEpiGroups = 2;            // epilogue warpgroups: one per accumulator, each taking every other tile
 constexpr int kEpiThreads = 128 * kEpiGroups;
@@ -56,17 +65,17 @@ struct ProjSmem {
     alignas(1024) unsigned char b[kPStages][kStageB];
     uint32_t list_key[kListCap][kEpiThreads];   // entry e of thread t at [e][t] (no bank conflicts): the logit as an ordered integer
     uint16_t list_col[kListCap][kEpiThreads];  // its column, counted from the first column of the CTA's part of the row block
-    uint64_t full[kPStages];         // the stage's operands have landed
+    uint64_t full[kPStages];         // (first CTA's) the stage's operands have landed in both CTAs
     uint64_t empty[kPStages];        // the stage's MMAs are done
     uint64_t acc_full[2];            // the accumulator holds a finished tile
-    uint64_t acc_empty[2];           // the epilogue has read the accumulator
+    uint64_t acc_empty[2];           // (first CTA's) the epilogues of both CTAs have read the accumulator
     uint32_t tmem_base;
     int abort_flag;
 };
 
 struct ProjParams {
     int R, V, D, K1;
-    int tiles_m, tiles_n;            // tiles along rows and along the vocabulary
+    int tiles_m, tiles_n;            // tiles (of a pair) along rows and along the vocabulary
     int pieces;                      // most pieces a row may have (stride of the per-piece arrays)
     ProjPieces out;
     uint32_t* row_tau;               // [R] zero before the launch: the highest bound any piece of the row has reached so far
@@ -79,9 +88,6 @@ __device__ __forceinline__ void pbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void pbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void pbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool pbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -103,10 +109,25 @@ __device__ __noinline__ bool pbar_wait(uint32_t bar, uint32_t parity, volatile i
     *abort_flag = 1;
     return false;
 }
-// 2-D tiled TMA load (no multicast): box at (x = element along the row, y = row) of the tensor map
+// 2-D tiled TMA load (no multicast): box at (x = element along the row, y = row) of the tensor map, into this CTA's
+// shared memory; the bytes are counted on `bar`, a shared::cluster address that may be the other CTA of the pair's
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// shared::cluster address of this CTA's shared-memory address `local` in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t local, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void pbar_arrive_cluster(uint32_t bar_cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 // Shared-memory operand descriptor of a K-major tile stored as rows of 128 bytes with the 128-byte swizzle:
 // start address, leading offset 1 (unused with a swizzle), 1024 bytes from one group of eight rows to the next,
@@ -120,18 +141,23 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
     d |= (uint64_t)2 << 61;
     return d;
 }
-// Instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 128, dense, no negation.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+// Instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 256 (the pair's), dense, no negation.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kPairM >> 4) << 24);
 
+// one MMA of the pair: the descriptors name the same shared-memory places in both CTAs, the accumulator the same
+// columns of both tensor memories; no output lane is masked
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+    const uint32_t zero = 0;
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(da), "l"(db), "r"(kIdesc), "r"(accumulate) : "memory");
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(kIdesc), "r"(accumulate), "r"(zero) : "memory");
 }
-// arrives on the mbarrier once every MMA issued so far by this thread has completed
+// arrives on the mbarrier at this place in both CTAs of the pair once every MMA issued so far by this thread has completed
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(both) : "memory");
 }
 __device__ __forceinline__ void tmem_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tmem_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -166,24 +192,28 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     volatile int* abort_flag = &sm.abort_flag;
 
-    // this CTA's run of tiles
+    // the pair, this CTA's place in it (0: the CTA that issues the MMAs and whose barriers count for both), and
+    // the pair's run of tiles
+    const uint32_t rank = cluster_rank();
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
-    const int t_begin = (int)((long long)blockIdx.x * n_tiles / gridDim.x);
-    const int t_end = (int)((long long)(blockIdx.x + 1) * n_tiles / gridDim.x);
+    const int t_begin = (int)((long long)pair * n_tiles / n_pairs);
+    const int t_end = (int)((long long)(pair + 1) * n_tiles / n_pairs);
     const int k_blocks = (p.D + kBK - 1) / kBK;
 
     if (tid == 0) {
         for (int s = 0; s < kPStages; ++s) { pbar_init(psmem_u32(&sm.full[s]), 1); pbar_init(psmem_u32(&sm.empty[s]), 1); }
-        for (int a = 0; a < 2; ++a) { pbar_init(psmem_u32(&sm.acc_full[a]), 1); pbar_init(psmem_u32(&sm.acc_empty[a]), 4); }
+        for (int a = 0; a < 2; ++a) { pbar_init(psmem_u32(&sm.acc_full[a]), 1); pbar_init(psmem_u32(&sm.acc_empty[a]), 2 * 4); }   // the four warps of one group in each CTA
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {       // tensor memory: the whole of it, for two accumulators
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(psmem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (warp == 1) {       // tensor memory: the whole of it in both CTAs (the same warp of each asks), for two accumulators
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(psmem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tmem_fence_before();
     __syncthreads();
+    cluster_sync_all();        // the other CTA's barriers exist before anything is signalled on them
     tmem_fence_after();
     const uint32_t tmem_base = sm.tmem_base;
 
@@ -201,20 +231,22 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 for (int kb = 0; kb < k_blocks; ++kb, ++n) {
                     const uint32_t s = n % kPStages, use = n / kPStages;
                     if (use > 0 && !pbar_wait(psmem_u32(&sm.empty[s]), (use - 1) & 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t bar = psmem_u32(&sm.full[s]);
-                    pbar_expect_tx(bar, kStageA + kStageB);
-                    tma_load_2d(psmem_u32(sm.a[s]), &map_a, kb * kBK, m * kBM, bar);
-                    tma_load_2d(psmem_u32(sm.b[s]), &map_b, kb * kBK, nn * kBN, bar);
+                    // both CTAs' bytes are counted on the first CTA's barrier, which that CTA arms
+                    if (rank == 0) pbar_expect_tx(psmem_u32(&sm.full[s]), 2 * (kStageA + kStageB));
+                    const uint32_t bar = cluster_addr(psmem_u32(&sm.full[s]), 0);
+                    tma_load_2d(psmem_u32(sm.a[s]), &map_a, kb * kBK, m * kPairM + (int)rank * kBM, bar);
+                    tma_load_2d(psmem_u32(sm.b[s]), &map_b, kb * kBK, nn * kBN + (int)rank * kHalfN, bar);
                 }
             }
-            if (!ok) {     // winding down: let the loads already issued land before the CTA leaves
+            // winding down: let the loads already issued (by both CTAs: the pair leaves together, after this) land
+            if (!ok && rank == 0) {
                 for (uint32_t f = n > kPStages ? n - kPStages : 0; f < n; ++f)
                     for (uint32_t i = 0; i < 100000 && !pbar_try_wait(psmem_u32(&sm.full[f % kPStages]), (f / kPStages) & 1u); ++i) {}
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer (first CTA of the pair)
+        if (lane == 0 && rank == 0) {
             uint32_t n = 0, tile_no = 0;
             bool ok = true;
 #pragma unroll 1
@@ -241,7 +273,8 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // ------------------------------------------------------------------ epilogue: a row of every other tile per thread
         const int et = tid - 128;                          // 0..255: place of this thread's list
         const int grp = (warp - 4) >> 2;                   // takes the tiles in accumulator grp (every other tile of the run)
-        const int trow = et & 127;                         // row of the tile = lane of tensor memory
+        const int trow = et & 127;                         // row of this CTA's half of the tile = lane of tensor memory
+        const int row_in_tile = (int)rank * kBM + trow;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         float cref = kPNoRef, sum = 0.f, tau = kTauNone;
         uint32_t tau_key = 0;              // tau as an ordered integer (0: none yet)
@@ -273,7 +306,7 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             // bound found.
             if (best > tau_key) {
                 tau_key = best;
-                if (cur_m * kBM + trow < p.R) atomicMax(p.row_tau + cur_m * kBM + trow, best);
+                if (cur_m * kPairM + row_in_tile < p.R) atomicMax(p.row_tau + cur_m * kPairM + row_in_tile, best);
             }
             best = tau_key;
             tau = tau_key ? unord32(tau_key) : kTauNone;
@@ -286,9 +319,9 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 }
             n_list = kept;
         };
-        auto flush = [&](int m, int piece) {      // write this thread's piece of row m * kBM + trow
+        auto flush = [&](int m, int piece) {      // write this thread's piece of row m * kPairM + row_in_tile
             compact();
-            const int row = m * kBM + trow;
+            const int row = m * kPairM + row_in_tile;
             if (row < p.R) {
                 if (lost) atomicOr(p.status, kStatusOverflow);
                 const int64_t slot = (int64_t)row * p.pieces + piece * kEpiGroups + grp;
@@ -301,13 +334,13 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 }
             }
         };
-        // piece of row block m that CTA c writes = c - (CTA that owns the row block's first tile)
+        // piece of row block m that pair c writes = c - (pair that owns the row block's first tile)
         auto first_cta = [&](int m) {
             const long long t0 = (long long)m * p.tiles_n;
             // largest c with c * n_tiles / grid <= t0
-            long long c = ((t0 + 1) * gridDim.x - 1) / n_tiles;
-            while (c > 0 && c * n_tiles / gridDim.x > t0) --c;
-            while ((c + 1) * n_tiles / gridDim.x <= t0) ++c;
+            long long c = ((t0 + 1) * n_pairs - 1) / n_tiles;
+            while (c > 0 && c * n_tiles / n_pairs > t0) --c;
+            while ((c + 1) * n_tiles / n_pairs <= t0) ++c;
             return (int)c;
         };
 
@@ -315,16 +348,16 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         for (int t = t_begin; t < t_end && ok; ++t, ++tile_no) {
             const int m = t / p.tiles_n, nn = t - m * p.tiles_n;
             if (m != cur_m) {          // (both groups pass here, whoever gets the row block's first tile)
-                if (cur_m >= 0) flush(cur_m, (int)blockIdx.x - first_cta(cur_m));
+                if (cur_m >= 0) flush(cur_m, pair - first_cta(cur_m));
                 cur_m = m; col_first = nn * kBN;
                 cref = kPNoRef; sum = 0.f; tau = kTauNone; tau_key = 0; n_list = 0; lost = false;
             }
             if ((tile_no & 1u) != (uint32_t)grp) continue;
             const uint32_t acc = (uint32_t)grp, acc_use = tile_no >> 1;
             // what the row's other pieces have found meanwhile (asked for before the wait, used after it)
-            const bool live = m * kBM + trow < p.R;            // (the last row block may reach past the last row)
+            const bool live = m * kPairM + row_in_tile < p.R;            // (the last row block may reach past the last row)
             uint32_t seen = 0;
-            if (live) asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(seen) : "l"(p.row_tau + m * kBM + trow));
+            if (live) asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(seen) : "l"(p.row_tau + m * kPairM + row_in_tile));
             // a list that has grown since its bound was last raised is tidied while the tile is still being computed
             if (__any_sync(kFullMask, n_list >= p.K1 + kRefreshSlack)) compact();
             if (!__all_sync(kFullMask, pbar_wait(psmem_u32(&sm.acc_full[acc]), acc_use & 1u, abort_flag))) { ok = false; break; }
@@ -400,15 +433,18 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             // the accumulator may be overwritten
             tmem_fence_before();
             __syncwarp();
-            if (lane == 0) pbar_arrive(psmem_u32(&sm.acc_empty[acc]));
+            if (lane == 0) pbar_arrive_cluster(cluster_addr(psmem_u32(&sm.acc_empty[acc]), 0));
         }
-        if (ok && cur_m >= 0) flush(cur_m, (int)blockIdx.x - first_cta(cur_m));
+        if (ok && cur_m >= 0) flush(cur_m, pair - first_cta(cur_m));
     }
+    // the pair leaves together: neither CTA's shared memory, barriers or tensor memory may go while the other
+    // could still signal or use them
     tmem_fence_before();
     __syncthreads();
+    cluster_sync_all();
     tmem_fence_after();
     if (warp == 1)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     if (tid == 0 && sm.abort_flag) atomicOr(p.status, kStatusTimeout);
 }
 
@@ -427,8 +463,8 @@ __global__ void __launch_bounds__(kMergeWarps * 32) project_merge_kernel(ProjPar
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     if (row >= p.R) return;
     const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
-    const int m = row / kBM;
-    // CTAs that own the first and the last tile of this row block
+    const int m = row / kPairM;
+    // pairs that own the first and the last tile of this row block
     auto owner = [&](long long t) {
         long long c = ((t + 1) * grid_scan - 1) / n_tiles;
         while (c > 0 && c * n_tiles / grid_scan > t) --c;
@@ -665,17 +701,18 @@ cudaError_t launch_constraint_logits(const void* hidden, int64_t hidden_stride, 
     return cudaGetLastError();
 }
 
-// CTAs of the scan: one per SM, more when a CTA would otherwise get more than kMaxRunTiles tiles
-static int project_grid(long long n_tiles, int sm_count) {
+// Pairs of CTAs of the scan: as many as can run at once, more when a pair would otherwise get more than
+// kMaxRunTiles tiles
+static int project_pairs(long long n_tiles, int max_pairs) {
     const long long by_run = (n_tiles + kMaxRunTiles - 1) / kMaxRunTiles;
-    const long long g = n_tiles < sm_count ? n_tiles : sm_count;
+    const long long g = n_tiles < max_pairs ? n_tiles : max_pairs;
     return (int)(g > by_run ? g : by_run);
 }
 
 int project_pieces(int R, int V, int sm_count) {
-    const int tiles_m = (R + kBM - 1) / kBM, tiles_n = (V + kBN - 1) / kBN;
-    const int grid = project_grid((long long)tiles_m * tiles_n, sm_count);
-    return ((grid + tiles_m - 1) / tiles_m + 2) * kEpiGroups;
+    const int tiles_m = (R + kPairM - 1) / kPairM, tiles_n = (V + kBN - 1) / kBN;
+    const int pairs = project_pairs((long long)tiles_m * tiles_n, sm_count / 2 > 0 ? sm_count / 2 : 1);
+    return ((pairs + tiles_m - 1) / tiles_m + 2) * kEpiGroups;
 }
 
 int project_list_cap() { return kListCap; }
@@ -685,29 +722,49 @@ bool project_scan_usable(const void* hidden, int64_t hidden_stride, const void* 
     return D >= 8 && D % 8 == 0 && K1 <= 32;
 }
 
-cudaError_t configure_project_scan() {
-    return cudaFuncSetAttribute(project_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ProjSmem) + 1024);
+static void pair_launch_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int pairs, cudaStream_t st) {
+    *cfg = cudaLaunchConfig_t{};
+    cfg->gridDim = dim3(2 * pairs, 1, 1); cfg->blockDim = dim3(kProjThreads, 1, 1);
+    cfg->dynamicSmemBytes = sizeof(ProjSmem) + 1024; cfg->stream = st;
+    attr->id = cudaLaunchAttributeClusterDimension;
+    attr->val.clusterDim.x = 2; attr->val.clusterDim.y = 1; attr->val.clusterDim.z = 1;
+    cfg->attrs = attr; cfg->numAttrs = 1;
+}
+
+// *max_pairs: how many pairs of CTAs the device runs at once (a pair needs two SMs of one GPC)
+cudaError_t configure_project_scan(int* max_pairs) {
+    cudaError_t e = cudaFuncSetAttribute(project_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ProjSmem) + 1024);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg; cudaLaunchAttribute attr;
+    pair_launch_config(&cfg, &attr, 1, nullptr);
+    int n = 0;
+    e = cudaOccupancyMaxActiveClusters(&n, project_scan_kernel, &cfg);
+    if (e != cudaSuccess) return e;
+    if (n < 1) return cudaErrorInvalidConfiguration;
+    *max_pairs = n;
+    return cudaSuccess;
 }
 
 cudaError_t launch_project_scan(const void* hidden, int64_t hidden_stride, const void* embed, int64_t embed_stride,
                                 int R, int V, int D, int K1, const ProjPieces& pieces, int piece_stride,
-                                const RowTop& top, uint32_t* status, int sm_count, cudaStream_t st, int* launches) {
+                                const RowTop& top, uint32_t* status, int max_pairs, cudaStream_t st, int* launches) {
     CUtensorMap map_a, map_b;
-    if (!make_map(&map_a, hidden, R, D, hidden_stride, kBM) || !make_map(&map_b, embed, V, D, embed_stride, kBN))
+    if (!make_map(&map_a, hidden, R, D, hidden_stride, kBM) || !make_map(&map_b, embed, V, D, embed_stride, kHalfN))
         return cudaErrorInvalidValue;
     ProjParams p;
     p.R = R; p.V = V; p.D = D; p.K1 = K1;
-    p.tiles_m = (R + kBM - 1) / kBM; p.tiles_n = (V + kBN - 1) / kBN;
+    p.tiles_m = (R + kPairM - 1) / kPairM; p.tiles_n = (V + kBN - 1) / kBN;
     p.pieces = piece_stride; p.out = pieces; p.row_tau = pieces.row_tau; p.status = status;
     cudaError_t e0 = cudaMemsetAsync(pieces.row_tau, 0, sizeof(uint32_t) * (size_t)R, st);
     if (e0 != cudaSuccess) return e0;
     const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
-    const int grid = project_grid(n_tiles, sm_count);
-    project_scan_kernel<<<grid, kProjThreads, sizeof(ProjSmem) + 1024, st>>>(map_a, map_b, p);
+    const int pairs = project_pairs(n_tiles, max_pairs);
+    cudaLaunchConfig_t cfg; cudaLaunchAttribute attr;
+    pair_launch_config(&cfg, &attr, pairs, st);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, project_scan_kernel, map_a, map_b, p);
     ++*launches;
-    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    project_merge_kernel<<<(R + kMergeWarps - 1) / kMergeWarps, kMergeWarps * 32, 0, st>>>(p, grid, top);
+    project_merge_kernel<<<(R + kMergeWarps - 1) / kMergeWarps, kMergeWarps * 32, 0, st>>>(p, pairs, top);
     ++*launches;
     return cudaGetLastError();
 }

@@ -157,6 +157,69 @@ def test_fused_projection_and_row_scan_match_the_oracle(dba, R, V, D, n_top):
         assert np.abs(X[r][idx[r]] - wv).max() <= tol, (r, idx[r], wi)
 
 
+def _bf16_pair(h, e):
+    from synth_inputs.logits import to_bf16_bits
+    hb, eb = to_bf16_bits(h), to_bf16_bits(e)
+    hd = torch.from_numpy(hb.view(np.int16)).cuda().view(torch.bfloat16)
+    ed = torch.from_numpy(eb.view(np.int16)).cuda().view(torch.bfloat16)
+    return hb, eb, hd, ed
+
+
+def test_fused_projection_long_runs_of_tiles(dba):
+    """Many row blocks and few CTAs per row block: a pair of CTAs works through a whole row block's vocabulary
+    (253 tiles), so the columns it keeps, counted from its first one, use all 16 bits.  Sampled rows against the
+    oracle (first and last rows, and rows on both sides of the boundaries between CTAs and between row blocks)."""
+    R, V, D, n_top = 19200, 64768, 16, 8
+    rng = np.random.default_rng(11)
+    h = rng.normal(0, 1, (R, D)).astype(np.float32)
+    e = rng.normal(0, 1, (V, D)).astype(np.float32)
+    e[-3:, :] = 3.0 * np.sign(h[R - 1])[None, :]              # the last row's best words are the vocabulary's last
+    hb, eb, hd, ed = _bf16_pair(h, e)
+    lse, val, idx = dba.project_scan(hd, ed, n_top)
+    lse, val, idx = lse.cpu().numpy(), val.cpu().numpy(), idx.cpu().numpy()
+    assert not np.isnan(lse).any()
+    rows = [0, 1, 127, 128, 255, 256, 9999, R - 129, R - 128, R - 1]
+    X = O.project(hb[rows], eb)
+    for i, r in enumerate(rows):
+        assert abs(float(lse[r]) - O.row_lse(X[i])) <= 1e-4
+        wv, wi = O.row_top(X[i], n_top)
+        assert np.abs(val[r] - wv).max() <= 1e-4
+        assert np.abs(X[i][idx[r]] - wv).max() <= 1e-4 and len(set(idx[r].tolist())) == n_top
+    assert set(idx[R - 1][:3].tolist()) == {V - 3, V - 2, V - 1}
+
+
+def test_fused_projection_ties_across_the_vocabulary(dba):
+    """Two hundred words spread over the vocabulary share a row's largest logit exactly: each thread meets only
+    a few of them, the merge of the row's pieces meets them all (more than its short list holds, and more
+    entries in all than it keeps in shared memory) and must list the lowest-numbered ones."""
+    R, V, D, n_top = 3, 64000, 8, 8
+    rng = np.random.default_rng(12)
+    h = np.zeros((R, D), np.float32); h[:, 0] = 1.0           # logits = embed[:, 0], exactly
+    e = np.zeros((V, D), np.float32)
+    e[:, 0] = np.clip(np.round(rng.normal(0, 1, V) * 8) / 16, -1.5, 1.5)      # (bf16-exact values below 2)
+    ties = 300 * np.arange(200) + 7
+    e[ties, 0] = 2.0
+    hb, eb, hd, ed = _bf16_pair(h, e)
+    lse, val, idx = dba.project_scan(hd, ed, n_top)
+    lse, val, idx = lse.cpu().numpy(), val.cpu().numpy(), idx.cpu().numpy()
+    X = O.project(hb, eb)
+    for r in range(R):
+        wv, wi = O.row_top(X[r], n_top)
+        assert np.array_equal(wi, ties[:n_top]) and np.array_equal(idx[r], wi) and np.array_equal(val[r], wv)
+        assert abs(float(lse[r]) - O.row_lse(X[r])) <= 1e-4
+
+
+def test_fused_projection_reports_a_plateau_it_cannot_hold(dba):
+    """Every logit of a row equal: a thread's list cannot hold the ties at the n_top-th largest value, and the
+    call reports it the documented way (every row NaN with an empty list) instead of listing a wrong choice."""
+    R, V, D, n_top = 4, 1000, 8, 5
+    h = np.zeros((R, D), np.float32)
+    e = np.ones((V, D), np.float32)
+    _, _, hd, ed = _bf16_pair(h, e)
+    lse, val, idx = dba.project_scan(hd, ed, n_top)
+    assert torch.isnan(lse).all() and (idx == -1).all() and torch.isinf(val).all()
+
+
 def test_fused_step_follows_the_oracle_on_the_projected_logits(dba):
     """dba_step_fused against the oracle stepping on the exactly projected logits.  Sentences must match field by
     field; where one first differs the two beams must hold the same scores rank by rank within the accumulated
