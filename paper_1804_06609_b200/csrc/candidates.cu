@@ -61,6 +61,8 @@ __host__ __device__ inline Layout make_layout(int k, int K1, int S, int max_cand
 // Merge of descending key lists of at most 32 entries each (key 0 = empty), one entry per lane: with the second
 // list reversed, the lane-wise maximum holds the 32 largest of both as a bitonic sequence, which five
 // compare-exchange steps put in descending order.
+constexpr int kMergeWays = 4;       // warps that share the merge of the row lists (source 1)
+
 __device__ __forceinline__ uint64_t merge_top32(uint64_t a, uint64_t b, int lane) {
     const uint64_t br = __shfl_sync(kFullMask, b, 31 - lane);
     uint64_t acc = a > br ? a : br;
@@ -109,6 +111,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     int* bank_cnt = reinterpret_cast<int*>(smem + L.bank_cnt);
     unsigned char* ent = smem + L.sort;
     __shared__ int s_ncand, s_ns1;
+    __shared__ uint64_t s_part[kMergeWays][32];       // partial merges of source 1
 
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -370,29 +373,37 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     __syncthreads();
 
     // ---- phase B (source 1): the k best cells of the whole matrix -----------------------------------------------
-    if (warp == 0 && k <= 32) {
-        // Every row's list is in (score desc, token asc) order and at most 32 long: the lists are merged one after
-        // the other, one entry per lane, with the bitonic top-32 merge; the first k of the result are the k best
-        // cells.  Keys: ordered score above, inverted flat index below (larger = better).
+    const int src1_warps = k <= 32 ? kMergeWays : 1;          // warps busy with source 1; the others take source 2
+    if (warp < kMergeWays && k <= 32) {
+        // Every row's list is in (score desc, token asc) order and at most 32 long: lists are merged, one entry
+        // per lane, with the bitonic top-32 merge -- every kMergeWays-th row by one of kMergeWays warps, then the
+        // partial results by the first of them; the first k of the result are the k best cells.
+        // Keys: ordered score above, inverted flat index below (larger = better).
         uint64_t acc = 0;
-        for (int h = 0; h < k; ++h) {
+        for (int h = warp; h < k; h += kMergeWays) {
             const uint64_t key = lane < rt_n[h]
                 ? ((uint64_t)ord32(rt_score[h * k + lane]) << 32) | (uint32_t)(0xffffffffu - (uint32_t)(h * V + rt_w[h * k + lane]))
                 : 0ull;
-            acc = h == 0 ? key : merge_top32(acc, key, lane);
+            acc = h == warp ? key : merge_top32(acc, key, lane);
         }
-        const bool have = lane < k && acc != 0ull;
-        const unsigned sel_mask = __ballot_sync(kFullMask, have);
-        const int flat = (int)(0xffffffffu - (uint32_t)acc);
-        const int h = have ? flat / V : -1 - lane;                       // (lanes without a cell match nobody)
-        // a row's cells are taken in its list's order: the cell's place in its row's list is the number of selected
-        // cells of the same row before it
-        const unsigned same = __match_any_sync(kFullMask, h) & sel_mask;
-        if (have) {
-            s1_h[lane] = h; s1_i[lane] = __popc(same & lt_mask);
-            atomicMax(&rt_ptr[h], __popc(same));
+        s_part[warp][lane] = acc;
+        asm volatile("bar.sync 1, %0;" ::"n"(kMergeWays * 32) : "memory");      // these warps only
+        if (warp == 0) {
+#pragma unroll
+            for (int w = 1; w < kMergeWays; ++w) acc = merge_top32(acc, s_part[w][lane], lane);
+            const bool have = lane < k && acc != 0ull;
+            const unsigned sel_mask = __ballot_sync(kFullMask, have);
+            const int flat = (int)(0xffffffffu - (uint32_t)acc);
+            const int h = have ? flat / V : -1 - lane;                       // (lanes without a cell match nobody)
+            // a row's cells are taken in its list's order: the cell's place in its row's list is the number of selected
+            // cells of the same row before it
+            const unsigned same = __match_any_sync(kFullMask, h) & sel_mask;
+            if (have) {
+                s1_h[lane] = h; s1_i[lane] = __popc(same & lt_mask);
+                atomicMax(&rt_ptr[h], __popc(same));
+            }
+            if (lane == 0) s_ns1 = __popc(sel_mask);
         }
-        if (lane == 0) s_ns1 = __popc(sel_mask);
     } else if (warp == 0) {
         // (beams wider than 32: a k-round tournament of row heads)
         // lane l holds the heads of rows l and l + 32: ordered score key and flat index of the best unused cell
@@ -430,7 +441,7 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
         //      raise its met count by one.  They all land in the same bank, so of one row at most k can ever be
         //      kept: with more, only the row's k best go on (the rest could not be selected; the bank still
         //      counts at least k candidates, which is all the allocation needs to know).
-        for (int h = warp - 1; h < k; h += n_warps - 1) {
+        for (int h = warp - src1_warps; h < k; h += n_warps - src1_warps) {
             if (s_kind[h] != 1) continue;
             const uint64_t m = s_mask[h];
             const float lse = s_lse[h], parent = s_parent[h];
