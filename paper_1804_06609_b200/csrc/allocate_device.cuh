@@ -72,6 +72,7 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
         int run = 0;                                  // exclusive prefix of n over banks, 32 at a time
 #pragma unroll
         for (int j = 0; j < 3; ++j) {
+            if (32 * j > C) break;                    // (no banks up there)
             int incl = nq[j];
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(kFullMask, incl, o); if (lane >= o) incl += t; }
@@ -125,6 +126,7 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
         int run = 0;
 #pragma unroll
         for (int j = 0; j < 3; ++j) {
+            if (32 * j > C) break;
             const int q = lane + 32 * j;
             const int a = q <= C ? alloc[q] : 0;
             int incl = a;
@@ -185,14 +187,25 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
     n_open = n_live - n_done;
     if (lane == 0 && n_open) list_base = atomicAdd(open_count, n_open);
     // new beam in decreasing score order, ties by lower flat index (Section 3.1), empty slots last
-    int open_before = 0;        // open cells handled in earlier rounds of the loop below
-    for (int i0 = 0; i0 < k; i0 += 32) {
+    static_assert(kMaxK <= 64, "a lane looks after at most two slots");
+    int slot_open[2] = {-1, -1};        // per round of the loop below: the row this lane's open cell went to, else -1
+#pragma unroll
+    for (int rd = 0; rd < 2; ++rd) {
+        const int i0 = 32 * rd;
+        if (i0 >= k) break;
         const int i = i0 + lane;
         const bool live = i < ns && !(pruning && a_val[i] < cut);
         int rank = 0, w = 0;
         if (live) {
             const float si = a_score[i]; const int fi = a_flat[i];
-            for (int j = 0; j < ns; ++j) rank += cell_better(a_score[j], a_flat[j], si, fi) && !(pruning && a_val[j] < cut);
+            // (branch-free and unrolled: the loads of several rounds are in flight together)
+            if (pruning) {
+#pragma unroll 8
+                for (int j = 0; j < ns; ++j) rank += (int)cell_better(a_score[j], a_flat[j], si, fi) & (int)!(a_val[j] < cut);
+            } else {
+#pragma unroll 8
+                for (int j = 0; j < ns; ++j) rank += (int)cell_better(a_score[j], a_flat[j], si, fi);
+            }
             const int id = sel[i];
             const uint64_t cmask = c_mask[id]; const int cactive = c_active[id];
             const int h = a_h[i];
@@ -210,12 +223,7 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
             if (out.met_mask) out.met_mask[r] = cmask;
             if (out.active) out.active[r] = cactive;
         }
-        // rows the next step has to scan: live slots that have not generated the end token
-        const bool open = live && w != d.eos_id;
-        const unsigned bal = __ballot_sync(kFullMask, open);
-        const int base = __shfl_sync(kFullMask, list_base, 0);
-        if (open) open_list[base + open_before + __popc(bal & ((1u << lane) - 1u))] = r0 + rank;
-        open_before += __popc(bal);
+        if (live && w != d.eos_id) slot_open[rd] = r0 + rank;
     }
     for (int i = n_live + lane; i < k; i += 32) {
         const int r = r0 + i;
@@ -228,6 +236,18 @@ __device__ __forceinline__ void allocate_sentence(const Dims& d, int b, int C, c
         if (out.bank) out.bank[r] = -1;
         if (out.met_mask) out.met_mask[r] = 0;
         if (out.active) out.active[r] = -1;
+    }
+    // rows the next step has to scan: live slots that have not generated the end token.  (Last, so that the reply
+    // to the reservation made above has had the whole of the beam's writing to arrive in.)
+    {
+        const int base = __shfl_sync(kFullMask, list_base, 0);
+        int open_before = 0;
+#pragma unroll
+        for (int rd = 0; rd < 2; ++rd) {
+            const unsigned bal = __ballot_sync(kFullMask, slot_open[rd] >= 0);
+            if (slot_open[rd] >= 0) open_list[base + open_before + __popc(bal & ((1u << lane) - 1u))] = slot_open[rd];
+            open_before += __popc(bal);
+        }
     }
     // Section 4's stopping rule (everything on the beam completed) and Section 6.4's early stopping (something is)
     if (out.stop && lane == 0)
