@@ -578,11 +578,12 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     }
     __syncthreads();
     {
-        // `split` neighbouring lanes share one candidate's count when there are threads to spare
-        int split = 1;
-        while (split < 8 && 2 * split * n <= n_threads) split <<= 1;
-        const int per_pass = n_threads / split;
-        for (int base = 0; base < n; base += per_pass) {
+        // `split` neighbouring lanes share one candidate's count when there are threads to spare (chosen pass by
+        // pass: the few candidates left for a last pass are counted by eight lanes each, not by one warp alone)
+        for (int base = 0, per_pass = 0; base < n; base += per_pass) {
+            int split = 1;
+            while (split < 8 && 2 * split * (n - base) <= n_threads) split <<= 1;
+            per_pass = n_threads / split;
             const int at = base + tid / split, part = tid & (split - 1);
             int rank = 0, lo = 0;
             uint32_t id = 0;
