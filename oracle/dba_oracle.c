@@ -105,7 +105,7 @@ double orc_row_lse(const void *row, int dtype, int V)
 }
 
 /* ------------------------------------------------------------------------------------------
- * Section 2, DECODER-STEP's last stage (Algorithm 1 line 4 produces the k x |V_T| matrix): the model output
+ * Section 2, DECODER-STEP's last stage (the step of Algorithm 1 that produces the k x |V_T| matrix): the model output
  * for hypothesis r and word w is the inner product of the decoder's final hidden state h_r with the
  * output embedding E_w.  Plain triple loop, bf16 inputs widened exactly, accumulation in double in
  * index order, one rounding to fp32 at the end.
