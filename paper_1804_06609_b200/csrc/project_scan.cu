@@ -9,7 +9,7 @@
 // has to fetch of the embedding, which is what bounds a single CTA on a 128 x 256 tile.  The tiles are numbered row
 // block by row block and dealt out to the pairs in equal contiguous runs, so a pair works through part of one row
 // block's vocabulary (and possibly the start of the next row block's).  Roles in each CTA, talking through mbarriers:
-//   warp 0    one thread issues the TMA loads (cp.async.bulk.tensor, cta_group::2, no multicast) of the 64-deep
+//   warp 0    one thread issues the TMA loads (cp.async.bulk.tensor, cta_group::2, each CTA for itself) of the 64-deep
 //             slices of this CTA's halves of both operands into a ring of shared-memory stages (128-byte swizzle);
 //             the bytes of both CTAs are counted on the first CTA's barrier;
 //   warp 1    allocates tensor memory (both CTAs); in the first CTA one thread issues the pair's tcgen05.mma
@@ -109,7 +109,7 @@ __device__ __noinline__ bool pbar_wait(uint32_t bar, uint32_t parity, volatile i
     *abort_flag = 1;
     return false;
 }
-// 2-D tiled TMA load (no multicast): box at (x = element along the row, y = row) of the tensor map, into this CTA's
+// 2-D tiled TMA load for this CTA alone: box at (x = element along the row, y = row) of the tensor map, into this CTA's
 // shared memory; the bytes are counted on `bar`, a shared::cluster address that may be the other CTA of the pair's
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
