@@ -21,7 +21,7 @@ __global__ void reset_kernel(Dims d, Beam beam, int32_t* __restrict__ open_list,
     beam.token[r] = first ? d.bos_id : d.pad_id;
     beam.mask[r] = 0; beam.active[r] = -1; beam.len[r] = 0; beam.bank[r] = first ? 0 : -1; beam.backptr[r] = 0;
     if (first) open_list[r / d.k] = r;
-    if (r == 0) *open_count = d.B;
+    if (r == 0) { open_count[0] = d.B; open_count[1] = 0; open_count[2] = 0; open_count[3] = 0; }   // counts of open rows, the row scan's work counters
 }
 
 // Section 3.3: the completed hypothesis with the highest score (Section 4: optionally divided by its

@@ -336,6 +336,8 @@ dba_status dba_step_fused(dba_handle* h, const void* hidden_dev, int64_t hidden_
     if (!step_events(h, &ev)) return DBA_ERR_CUDA;
     // the list of open rows is not used by this path (every row is projected), but its count is kept in step
     cudaError_t e = cudaMemsetAsync(h->open_count + ((h->t + 1) & 1), 0, sizeof(int32_t), h->stream);
+    // (nor does it run the row scan, whose launches clear each other's work counter in turn: both are cleared here)
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->open_count + 2, 0, 2 * sizeof(int32_t), h->stream);
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[0], h->stream);
     if (e == cudaSuccess)
         e = launch_project_scan(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, h->d.R, h->d.V, D, h->d.K1,

@@ -19,6 +19,7 @@ constexpr uint32_t kStatusOverflow = 2u;   // an internal list ran out of room (
 // further words of the status block: counters (diagnostics, never an error)
 constexpr int kStatusWordRescans = 1;      // stretches of rows the scan kernel had to rank from global memory again
 constexpr int kStatusWordUnresolved = 2;   // fused step: rows whose equal scores ran past the row's list and could not be looked up
+constexpr int kStatusWordTicket = 4;       // stand-alone row scan: the counter its CTAs draw their items from (cleared with the block)
 
 // Per-sentence constraint table, phrases flattened to token positions 0..C-1 (Section 3 of the paper:
 // the constraint count is the total number of tokens over all words and phrases).

@@ -57,6 +57,10 @@ struct WaitCtl {
     long long wait_clocks;                  // how long a wait may last
 };
 
+constexpr int kStaticItems = kSlots;         // a CTA's first items are fixed by its number, the rest drawn from a counter
+constexpr int kItemRing = 4 * kSlots;        // item descriptors kept in shared memory
+struct ItemDesc { int row; int seg; };       // what the producer tells the other roles about an item; row < 0: no more items
+
 struct Smem {
     alignas(128) unsigned char ring[kSlots][kTeamWarps * kChunkBytes];
     alignas(16) uint4 cell_max[kSlots][kTeamWarps][32];     // per lane: the maxima of its four pairs of vectors
@@ -76,6 +80,7 @@ struct Smem {
     int hit[kSlots][2][kHitCap];            // cells that reach the bound: (first vector of the pair) * 2 + parity
     int hit_n[kSlots][2];                   // how many (above kHitCap: the list overflowed)
     float hit_bound[kSlots][2];
+    ItemDesc item[kItemRing];               // by item number % kItemRing
     WaitCtl ctl;
 };
 
@@ -87,6 +92,8 @@ struct Params {
     const int32_t* open_list;   // rows to scan (null: all R rows)
     const int32_t* open_count;  // number of entries of open_list (device memory)
     int32_t* zero_count;        // set to zero here: the count of the list the step's last kernel builds (may be null)
+    int32_t* ticket;            // zero at launch: the counter the CTAs draw their items from
+    int32_t* zero_ticket;       // set to zero here: the next launch's counter (may be null)
     float* part_m; float* part_s; float* top_val; int32_t* top_idx;     // results, per (row, segment)
     uint32_t* status;
     long long wait_clocks;      // how long a wait may last
@@ -222,20 +229,27 @@ template <> struct Vec<__nv_bfloat16> {
     }
 };
 
-// The items of this CTA, in the order all roles agree on.
-// Items are numbered row-major over (position in the list of open rows, segment); this CTA takes every
-// gridDim.x-th one.  The walk needs no division after the constructor.
+// Which item is whose.  Items are numbered row-major over (position in the list of open rows, segment).  A CTA's
+// first kStaticItems items are fixed by its number (item c + n * gridDim.x for its n-th), so that it can start
+// without asking; the rest are drawn one at a time from a counter in global memory, so that a CTA that gets ahead
+// (the memory system does not serve all SMs alike from one launch to the next: CTAs given equal shares finish up
+// to 10 us apart) takes more.  The producer draws (kStaticItems items ahead of the copy it issues), looks the row up and
+// leaves (row, segment) in a ring of descriptors in shared memory, where the other roles find it after the wait
+// that orders them behind the producer; a descriptor without a row says that there are no more items.  It is
+// written for the item of each of the kSlots buffers after the last, passes through all roles like an item
+// without data, and each role stops when it has met as many as it serves buffers.
+// A descriptor is overwritten kItemRing items later, which the copy into the same buffer three uses later waits
+// for: by then the buffer's ranking warp, the last to look at it, has finished the buffer's next item.
+
+// A role's place in its CTA's sequence of items, and the geometry of the item it is at.
 // (Only a row's last segment differs from the others in length: what depends on the length alone -- bytes, chunks,
 // the tap of the reports -- is worked out once for the two kinds, and an item picks one.)
 struct ItemIter {
-    int i, seg_, n_rows, S, step_i, step_seg;
+    int S, seg_, row_;
     int bytes_kind[2], chunks_kind[2], tap_kind[2];     // [0]: a full segment, [1]: the row's last segment
     int bytes_, n_chunks_, tap_;  // of the current item
     uint32_t n_item;
-    __device__ ItemIter(const Params& p, int elem_bytes) : S(p.S), n_item(0) {
-        n_rows = p.open_count ? *p.open_count : p.R;
-        i = blockIdx.x / S; seg_ = blockIdx.x - i * S;
-        step_i = gridDim.x / S; step_seg = gridDim.x - step_i * S;
+    __device__ ItemIter(const Params& p, int elem_bytes) : S(p.S), seg_(0), row_(-1), n_item(0) {
         const int seg_bytes_full = p.seg_len * elem_bytes, row_bytes = p.V * elem_bytes;
         bytes_kind[0] = seg_bytes_full;
         bytes_kind[1] = row_bytes - (S - 1) * seg_bytes_full;
@@ -244,28 +258,20 @@ struct ItemIter {
             chunks_kind[q] = (bytes_kind[q] + kChunkBytes - 1) / kChunkBytes;
             tap_kind[q] = tap_for(bytes_kind[q], p.K1);
         }
-        load();
+        set(-1, 0);
     }
-    __device__ __forceinline__ void load() {
+    __device__ __forceinline__ void set(int row, int seg) {
+        row_ = row; seg_ = seg;
         const bool last = seg_ == S - 1;
         bytes_ = last ? bytes_kind[1] : bytes_kind[0];
         n_chunks_ = last ? chunks_kind[1] : chunks_kind[0];
         tap_ = last ? tap_kind[1] : tap_kind[0];
     }
-    __device__ bool valid() const { return i < n_rows; }
-    __device__ void next() {
-        n_item += 1;
-        i += step_i; seg_ += step_seg;
-        if (seg_ >= S) { seg_ -= S; ++i; }
-        load();
-    }
-    __device__ void skip(int k) {       // k times next()
-        n_item += (uint32_t)k;
-        i += k * step_i; seg_ += k * step_seg;
-        while (seg_ >= S) { seg_ -= S; ++i; }
-        load();
-    }
-    __device__ int row(const int32_t* open_list) const { return open_list ? __ldg(open_list + i) : i; }
+    // the descriptor the producer left for this item (call after the wait that orders this role behind it)
+    __device__ __forceinline__ void fetch(const ItemDesc* ring) { const ItemDesc d = ring[n_item % kItemRing]; set(d.row, d.seg); }
+    __device__ bool valid() const { return row_ >= 0; }
+    __device__ void skip(int k) { n_item += (uint32_t)k; }
+    __device__ int row() const { return row_; }
     __device__ int seg() const { return seg_; }
     __device__ int bytes() const { return bytes_; }
     __device__ int n_chunks() const { return n_chunks_; }
@@ -337,37 +343,64 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
     grid_dependency_wait();      // the list of open rows comes from the previous step's last kernel
     if (tid == 0) {
         if (blockIdx.x == 0 && p.zero_count) *p.zero_count = 0;     // before the next kernel can start
+        if (blockIdx.x == 0 && p.zero_ticket) *p.zero_ticket = 0;
         allow_dependents();
     }
 
     if (warp == kWarpProd) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            ItemIter it(p, (int)sizeof(T)), ahead = it;
+            ItemIter it(p, (int)sizeof(T));
             bool ok = true;
-            // the row numbers come from a list in global memory: they are asked for kSlots items ahead, so that
-            // no copy waits for one (the first kSlots loads overlap one another, and the load of the list's length:
-            // a place beyond the length is still a place of the list, its value is just not used)
-            int rows[kSlots];
+            // Items are drawn 2 * kAhead items ahead and their rows looked up kAhead ahead (the list of open rows is in
+            // global memory), so that no copy waits for either, and no further, so that a CTA is committed to few
+            // items when the counter runs out: g_far[q] is the number of the item 2 * kAhead from now, g_near[q] /
+            // row_near[q] number and row of the item kAhead from now (q = item number % kAhead).  The first loads
+            // overlap the load of the list's length: a place beyond the length is still a place of the list, its
+            // value is just not used.
+            const int S = p.S;
+            auto row_of = [&](int g) { const int i = g / S; return i < p.R ? (p.open_list ? __ldg(p.open_list + i) : i) : 0; };
+            constexpr int kAhead = kStaticItems / 2;
+            static_assert(kSlots % kAhead == 0, "the queues are indexed by the buffer number");
+            int g_near[kAhead], row_near[kAhead], g_far[kAhead];
 #pragma unroll
-            for (int j = 0; j < kSlots; ++j) { rows[j] = ahead.i < p.R ? ahead.row(p.open_list) : 0; ahead.next(); }
+            for (int q = 0; q < kAhead; ++q) {
+                g_near[q] = (int)blockIdx.x + q * (int)gridDim.x; row_near[q] = row_of(g_near[q]);
+                g_far[q] = (int)blockIdx.x + (kAhead + q) * (int)gridDim.x;
+            }
+            const int n_rows = p.open_count ? *p.open_count : p.R;
+            const int total = n_rows * S;                 // items of this launch
+            int n_end = 0;                                // descriptors without a row written so far
 #pragma unroll 1
-            while (ok && it.valid()) {
+            while (ok && n_end < kSlots) {
 #pragma unroll
                 for (int j = 0; j < kSlots; ++j) {          // item n uses slot n % kSlots = j
-                    if (!it.valid()) break;
+                    if (n_end == kSlots) break;
                     const uint32_t slot = j;
-                    const int row = rows[j];
-                    rows[j] = ahead.i < p.R ? ahead.row(p.open_list) : 0;
-                    ahead.next();
-                    if (!mbar_try_wait(smem_u32(&sm.loaded[slot]), it.slot_phase() ^ 1u) &&
-                        !mbar_wait(smem_u32(&sm.loaded[slot]), it.slot_phase() ^ 1u, abort_flag)) { ok = false; break; }
-                    const char* src = (const char*)p.logits + ((int64_t)row * p.stride + (int64_t)it.seg() * p.seg_len) * (int64_t)sizeof(T);
-                    mbar_expect_tx(smem_u32(&sm.full[slot]), (uint32_t)it.bytes());
-                    if ((int)it.n_item != p.drop_item)
-                        bulk_load(smem_u32(sm.ring[slot]), src, (uint32_t)it.bytes(), smem_u32(&sm.full[slot]));
-                    it.next();
-                    sm.ctl.n_issued = it.n_item;
+                    const int q = j % kAhead;              // (a constant once the loop is unrolled)
+                    const int g = g_near[q], row = row_near[q];
+                    g_near[q] = g_far[q]; row_near[q] = row_of(g_far[q]);
+                    g_far[q] = kStaticItems * (int)gridDim.x + atomicAdd(p.ticket, 1);
+                    const uint32_t phase = (it.n_item / kSlots) & 1u;
+                    if (!mbar_try_wait(smem_u32(&sm.loaded[slot]), phase ^ 1u) &&
+                        !mbar_wait(smem_u32(&sm.loaded[slot]), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    ItemDesc* desc = &sm.item[it.n_item % kItemRing];
+                    if (g < total) {
+                        const int seg = g - (g / S) * S;
+                        it.set(row, seg);
+                        desc->row = row; desc->seg = seg;
+                        const char* src = (const char*)p.logits + ((int64_t)row * p.stride + (int64_t)seg * p.seg_len) * (int64_t)sizeof(T);
+                        mbar_expect_tx(smem_u32(&sm.full[slot]), (uint32_t)it.bytes());
+                        if ((int)it.n_item != p.drop_item)
+                            bulk_load(smem_u32(sm.ring[slot]), src, (uint32_t)it.bytes(), smem_u32(&sm.full[slot]));
+                        it.skip(1);
+                        sm.ctl.n_issued = it.n_item;
+                    } else {            // no more items: an item without data, for the roles that serve this buffer to stop at
+                        desc->row = -1; desc->seg = 0;
+                        mbar_arrive(smem_u32(&sm.full[slot]));
+                        it.skip(1);
+                        ++n_end;
+                    }
                 }
             }
         }
@@ -376,16 +409,25 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
         // ------------------------------------------------------------------ consumers
         const int team = (warp - kWarpCons) / kTeamWarps, chunk = (warp - kWarpCons) - team * kTeamWarps;
         ItemIter it(p, (int)sizeof(T));
+        int n_ends = 0;                            // items without data met: one for each of the team's kSlots / kTeams buffers
 #pragma unroll 1
-        for (it.skip(team); it.valid(); it.skip(kTeams)) {
+        for (it.skip(team);; it.skip(kTeams)) {
             const uint32_t slot = it.slot(), half = it.use() & 1u;
-            const int nvec = chunk < it.n_chunks() ? it.chunk_vecs(chunk) : 0;
             uint4 v[kVecsPerLane];
             typename Vec<T>::Max pmax[kPairs];
             uint32_t key = 0;                      // below the key of every value, -inf included
             // A warp without a chunk in this item waits for the copy all the same: it must not run ahead and sign
             // the buffer off (`loaded`) for this use while a slower warp has yet to do so for the previous one.
             if (!mbar_wait_warp(smem_u32(&sm.full[slot]), it.slot_phase(), abort_flag)) break;
+            it.fetch(sm.item);
+            if (!it.valid()) {
+                // no more items: the word is passed on to the buffer's selector, in turn like any item's reports
+                if (!mbar_wait_warp(smem_u32(&sm.slot_free[slot]), it.slot_phase() ^ 1u, abort_flag)) break;
+                if (lane == 0) mbar_arrive(smem_u32(&sm.reports_in[slot]));
+                if (++n_ends == kSlots / kTeams) break;
+                continue;
+            }
+            const int nvec = chunk < it.n_chunks() ? it.chunk_vecs(chunk) : 0;
             if (nvec > 0) {
                 const uint4* vec = reinterpret_cast<const uint4*>(sm.ring[slot]) + chunk * kChunkVecs + lane;
                 if (nvec >= kChunkVecs) {
@@ -459,8 +501,14 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
         ItemIter it(p, (int)sizeof(T));
         it.skip(rk);                                      // this selector's first item
 #pragma unroll 1
-        while (it.valid()) {
+        for (;;) {
             if (!mbar_wait_warp(smem_u32(&sm.reports_in[slot]), it.slot_phase(), abort_flag)) break;
+            it.fetch(sm.item);
+            if (!it.valid()) {                            // no more items: tell the ranking warp, in turn
+                if (!mbar_wait_warp(smem_u32(&sm.ranked[slot]), it.slot_phase() ^ 1u, abort_flag)) break;
+                if (lane == 0) mbar_arrive(smem_u32(&sm.hits_ready[slot]));
+                break;
+            }
             // The bound: the K1-th largest report, i.e. the largest report that at least K1 reports reach.
             const uint32_t half = it.use() & 1u;
             int* hits = sm.hit[slot][half];
@@ -579,11 +627,13 @@ __global__ void __launch_bounds__(kThreads, 1) row_scan_tma_kernel(Params p) {
         ItemIter it(p, (int)sizeof(T));
         it.skip(rk);
 #pragma unroll 1
-        while (it.valid()) {
-            const int row = it.row(p.open_list);
+        for (;;) {
+            if (!mbar_wait_warp(smem_u32(&sm.hits_ready[slot]), it.slot_phase(), abort_flag)) break;
+            it.fetch(sm.item);
+            if (!it.valid()) break;                       // no more items
+            const int row = it.row();
             const uint32_t half = it.use() & 1u, use_phase = (it.use() >> 1) & 1u;
             const int nc = it.n_chunks();
-            if (!mbar_wait_warp(smem_u32(&sm.hits_ready[slot]), it.slot_phase(), abort_flag)) break;
             const int* hits = sm.hit[slot][half];
             const int nh = sm.hit_n[slot][half];
             const float tau = sm.hit_bound[slot][half];
@@ -712,6 +762,11 @@ cudaError_t launch_row_scan_tma(const void* logits, int64_t stride, const Dims& 
     Params p;
     p.logits = logits; p.stride = stride; p.V = d.V; p.S = d.S; p.seg_len = d.seg_len; p.K1 = d.K1; p.R = d.R;
     p.open_list = open_list; p.open_count = open_count; p.zero_count = zero_count;
+    // the work counter: with a list of open rows, the word two places after its count (the step alternates between
+    // two counts, and so between two counters: each launch clears the other's); else a word of the status block,
+    // which the caller has just cleared
+    p.ticket = open_count ? const_cast<int32_t*>(open_count) + 2 : reinterpret_cast<int32_t*>(status) + kStatusWordTicket;
+    p.zero_ticket = open_count && zero_count ? zero_count + 2 : nullptr;
     p.part_m = part.m; p.part_s = part.s; p.top_val = part.val; p.top_idx = part.idx; p.status = status;
     p.wait_clocks = dbg.wait_clocks > 0 ? dbg.wait_clocks : 2000000000LL;       // about a second: a wait this long has failed
     p.drop_item = dbg.drop_item;
