@@ -30,6 +30,7 @@ struct dba_handle {
     uint32_t* status;
     int32_t* open_list;            // rows the next step scans, and how many
     int32_t* open_count;           // two counts: step t reads [t & 1], its last kernel fills [(t + 1) & 1]
+                                   // ([2], [3]: the row scan's work counters, alternating the same way)
     int32_t* fin_tokens; int32_t* fin_len; float* fin_score; int32_t* fin_flags;
     void* stage_logits;            // only with DBA_FLAG_HOST_STAGING
     dba_step_out stage_out;
