@@ -228,7 +228,11 @@ uint64_t dba_launch_count(const dba_handle* h);
  *   drop_item    >= 0: every thread block announces the copy of this item (a stretch of up to 44 KB of a row) of
  *                its sequence but does not issue it, so the wait for it runs out after wait_clocks; the kernel
  *                then records the failure and returns (nothing faults or hangs).  < 0: every copy is issued.
- * h == NULL sets the two for the stand-alone scans of this process (dba_row_scan, dba_row_scan_static).
+ * The fused projection (dba_step_fused, dba_project_scan) takes the same two: there the item is a 64-deep slice
+ * of the operands in the sequence of the first thread block of every pair, which announces its copies of that
+ * slice without issuing them; both blocks of the pair then give up at their next wait and leave together.
+ * h == NULL sets the two for the stand-alone scans of this process (dba_row_scan, dba_row_scan_static,
+ * dba_project_scan).
  */
 dba_status dba_test_hook(dba_handle* h, int64_t wait_clocks, int32_t drop_item);
 

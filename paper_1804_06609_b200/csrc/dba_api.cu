@@ -342,7 +342,7 @@ dba_status dba_step_fused(dba_handle* h, const void* hidden_dev, int64_t hidden_
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[0], h->stream);
     if (e == cudaSuccess)
         e = launch_project_scan(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, h->d.R, h->d.V, D, h->d.K1,
-                                h->proj, h->proj_stride, h->top, h->status, h->proj_pairs, h->stream, &h->launches_tmp);
+                                h->proj, h->proj_stride, h->top, h->status, h->proj_pairs, h->dbg, h->stream, &h->launches_tmp);
     if (ev && e == cudaSuccess) e = cudaEventRecord(ev[1], h->stream);
     if (e == cudaSuccess)
         e = launch_constraint_logits(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, D, h->d, h->cons,
@@ -563,7 +563,7 @@ dba_status dba_project_scan(const void* hidden_dev, int64_t hidden_stride_elems,
     if (e == cudaSuccess) e = configure_project_scan(&max_pairs);
     if (e == cudaSuccess)
         e = launch_project_scan(hidden_dev, hidden_stride_elems, embed_dev, embed_stride_elems, R, V, D, n_top, pieces, stride,
-                                top, status, max_pairs, stream, &launches);
+                                top, status, max_pairs, g_scan_debug, stream, &launches);
     if (e == cudaSuccess) e = launch_scan_check(status, R, n_top, top, stream);
     return cuda_fail(e);
 }

@@ -83,10 +83,11 @@ struct ProjPieces {
     uint32_t* row_tau; // [R] the bound the row's pieces share while the kernel runs (an ordered integer; zeroed per launch)
 };
 
-// Testing aids of the streaming scan (see dba_test_hook in dba.h).
+// Testing aids of the streaming scan and of the fused projection (see dba_test_hook in dba.h).
 struct ScanDebug {
     long long wait_clocks = 0;   // > 0: how many clocks a wait on an mbarrier may last
-    int drop_item = -1;          // >= 0: every CTA announces the copy of this item of its sequence but never issues it
+    int drop_item = -1;          // >= 0: every CTA (projection: the first of every pair) announces the copy of this item
+                                 //       of its sequence but never issues it
 };
 
 // How the candidate kernel is launched for one handle: fixed at dba_init from the handle's own device.
@@ -141,7 +142,7 @@ bool project_scan_usable(const void* hidden, int64_t hidden_stride, const void* 
 cudaError_t configure_project_scan(int* max_pairs);      // *max_pairs: pairs of CTAs the device runs at once
 cudaError_t launch_project_scan(const void* hidden, int64_t hidden_stride, const void* embed, int64_t embed_stride,
                                 int R, int V, int D, int K1, const ProjPieces& pieces, int piece_stride,
-                                const RowTop& top, uint32_t* status, int max_pairs, cudaStream_t st, int* launches);
+                                const RowTop& top, uint32_t* status, int max_pairs, const ScanDebug& dbg, cudaStream_t st, int* launches);
 // logits of every sentence's constraint tokens for its rows: out[r * 64 + j] = <hidden[r], embed[token j of the
 // sentence of row r]> (fp32), for the fused step, which has no logit matrix to look them up in
 cudaError_t launch_constraint_logits(const void* hidden, int64_t hidden_stride, const void* embed, int64_t embed_stride,

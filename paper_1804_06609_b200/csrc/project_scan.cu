@@ -58,7 +58,12 @@ constexpr int kRefreshSlack = 8;         // arrivals beyond K1 after which a lis
 constexpr int kMaxRunTiles = 256;        // tiles a CTA may work through: columns are kept relative to its first one, in 16 bits
 constexpr int kProjThreads = 128 + kEpiThreads;
 constexpr int kTmemCols = 512;           // two accumulators of 256 columns
-constexpr long long kProjWaitClocks = 4000000000LL;      // about two seconds: a wait this long has failed
+constexpr long long kProjWaitClocks = 4000000000LL;      // about two seconds: a wait this long has failed (the default)
+
+struct ProjWait {
+    int abort_flag;                  // a wait has run out: every role leaves at its next wait
+    long long wait_clocks;           // how long a wait may last
+};
 
 struct ProjSmem {
     alignas(1024) unsigned char a[kPStages][kStageA];
@@ -70,7 +75,7 @@ struct ProjSmem {
     uint64_t acc_full[2];            // the accumulator holds a finished tile
     uint64_t acc_empty[2];           // (first CTA's) the epilogues of both CTAs have read the accumulator
     uint32_t tmem_base;
-    int abort_flag;
+    ProjWait ctl;
 };
 
 struct ProjParams {
@@ -80,6 +85,8 @@ struct ProjParams {
     ProjPieces out;
     uint32_t* row_tau;               // [R] zero before the launch: the highest bound any piece of the row has reached so far
     uint32_t* status;
+    long long wait_clocks;           // how long a wait may last
+    int drop_item;                   // testing: the first CTA of every pair announces the copies of this slice of its sequence but never issues them
 };
 
 __device__ __forceinline__ uint32_t psmem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -97,16 +104,17 @@ __device__ __forceinline__ bool pbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  False: the CTA is winding down (this wait ran out, or another one did).
-__device__ __noinline__ bool pbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __noinline__ bool pbar_wait(uint32_t bar, uint32_t parity, volatile ProjWait* ctl) {
+    const long long limit = ctl->wait_clocks;
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 32; ++i)
             if (pbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kProjWaitClocks) break;
+        if (ctl->abort_flag) return false;
+        if (clock64() - t0 > limit) break;
     }
-    *abort_flag = 1;
+    ctl->abort_flag = 1;
     return false;
 }
 // 2-D tiled TMA load for this CTA alone: box at (x = element along the row, y = row) of the tensor map, into this CTA's
@@ -190,7 +198,7 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // the operand tiles want 1024-byte alignment (the swizzle pattern repeats every 1024 bytes)
     ProjSmem& sm = *reinterpret_cast<ProjSmem*>(psmem_raw + ((1024u - (psmem_u32(psmem_raw) & 1023u)) & 1023u));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    volatile int* abort_flag = &sm.abort_flag;
+    volatile ProjWait* abort_flag = &sm.ctl;
 
     // the pair, this CTA's place in it (0: the CTA that issues the MMAs and whose barriers count for both), and
     // the pair's run of tiles
@@ -204,7 +212,7 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     if (tid == 0) {
         for (int s = 0; s < kPStages; ++s) { pbar_init(psmem_u32(&sm.full[s]), 1); pbar_init(psmem_u32(&sm.empty[s]), 1); }
         for (int a = 0; a < 2; ++a) { pbar_init(psmem_u32(&sm.acc_full[a]), 1); pbar_init(psmem_u32(&sm.acc_empty[a]), 2 * 4); }   // the four warps of one group in each CTA
-        sm.abort_flag = 0;
+        sm.ctl.abort_flag = 0; sm.ctl.wait_clocks = p.wait_clocks;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {       // tensor memory: the whole of it in both CTAs (the same warp of each asks), for two accumulators
@@ -234,14 +242,17 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     // both CTAs' bytes are counted on the first CTA's barrier, which that CTA arms
                     if (rank == 0) pbar_expect_tx(psmem_u32(&sm.full[s]), 2 * (kStageA + kStageB));
                     const uint32_t bar = cluster_addr(psmem_u32(&sm.full[s]), 0);
+                    if (rank == 0 && (int)n == p.drop_item) continue;
                     tma_load_2d(psmem_u32(sm.a[s]), &map_a, kb * kBK, m * kPairM + (int)rank * kBM, bar);
                     tma_load_2d(psmem_u32(sm.b[s]), &map_b, kb * kBK, nn * kBN + (int)rank * kHalfN, bar);
                 }
             }
             // winding down: let the loads already issued (by both CTAs: the pair leaves together, after this) land
             if (!ok && rank == 0) {
-                for (uint32_t f = n > kPStages ? n - kPStages : 0; f < n; ++f)
+                for (uint32_t f = n > kPStages ? n - kPStages : 0; f < n; ++f) {
+                    if ((int)f == p.drop_item) continue;
                     for (uint32_t i = 0; i < 100000 && !pbar_try_wait(psmem_u32(&sm.full[f % kPStages]), (f / kPStages) & 1u); ++i) {}
+                }
             }
         }
     } else if (warp == 1) {
@@ -445,7 +456,7 @@ project_scan_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     tmem_fence_after();
     if (warp == 1)
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-    if (tid == 0 && sm.abort_flag) atomicOr(p.status, kStatusTimeout);
+    if (tid == 0 && sm.ctl.abort_flag) atomicOr(p.status, kStatusTimeout);
 }
 
 // Orders the pieces of every row exactly: one warp per row adds up the pieces' sums (in the order of the pieces),
@@ -462,6 +473,9 @@ __global__ void __launch_bounds__(kMergeWarps * 32) project_merge_kernel(ProjPar
     const int row = blockIdx.x * kMergeWarps + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     if (row >= p.R) return;
+    // a scan that gave up (a wait that ran out, a list that overflowed) has not written every piece: nothing is
+    // read, the row's results stay what they were, and the failure is reported from the status word
+    if (*reinterpret_cast<volatile uint32_t*>(p.status) & (kStatusTimeout | kStatusOverflow)) return;
     const long long n_tiles = (long long)p.tiles_m * p.tiles_n;
     const int m = row / kPairM;
     // pairs that own the first and the last tile of this row block
@@ -747,7 +761,8 @@ cudaError_t configure_project_scan(int* max_pairs) {
 
 cudaError_t launch_project_scan(const void* hidden, int64_t hidden_stride, const void* embed, int64_t embed_stride,
                                 int R, int V, int D, int K1, const ProjPieces& pieces, int piece_stride,
-                                const RowTop& top, uint32_t* status, int max_pairs, cudaStream_t st, int* launches) {
+                                const RowTop& top, uint32_t* status, int max_pairs, const ScanDebug& dbg, cudaStream_t st,
+                                int* launches) {
     CUtensorMap map_a, map_b;
     if (!make_map(&map_a, hidden, R, D, hidden_stride, kBM) || !make_map(&map_b, embed, V, D, embed_stride, kHalfN))
         return cudaErrorInvalidValue;
@@ -755,6 +770,7 @@ cudaError_t launch_project_scan(const void* hidden, int64_t hidden_stride, const
     p.R = R; p.V = V; p.D = D; p.K1 = K1;
     p.tiles_m = (R + kPairM - 1) / kPairM; p.tiles_n = (V + kBN - 1) / kBN;
     p.pieces = piece_stride; p.out = pieces; p.row_tau = pieces.row_tau; p.status = status;
+    p.wait_clocks = dbg.wait_clocks > 0 ? dbg.wait_clocks : kProjWaitClocks; p.drop_item = dbg.drop_item;
     cudaError_t e0 = cudaMemsetAsync(pieces.row_tau, 0, sizeof(uint32_t) * (size_t)R, st);
     if (e0 != cudaSuccess) return e0;
     const long long n_tiles = (long long)p.tiles_m * p.tiles_n;

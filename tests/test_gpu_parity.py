@@ -672,6 +672,39 @@ def test_a_device_wait_that_runs_out_is_reported_and_the_device_stays_usable(dba
     st2.close()
 
 
+def test_a_wait_that_runs_out_in_the_fused_projection_is_reported(dba):
+    """The same for the projection kernel, whose pairs of CTAs wait on each other's copies: the first CTA of every
+    pair announces its first slice of the operands without fetching it, the limit is about a millisecond, every
+    role of both CTAs gives up at its next wait and the pair leaves together.  The stand-alone call reports NaN
+    rows; the fused step's dba_finalize reports DBA_ERR_TIMEOUT; afterwards the same calls work."""
+    R, V, D, n_top = 300, 5000, 128, 7
+    rng = np.random.default_rng(5)
+    h = rng.normal(0, 1, (R, D)).astype(np.float32)
+    e = rng.normal(0, 1, (V, D)).astype(np.float32)
+    _, _, hd, ed = _bf16_pair(h, e)
+    L = dba.lib()
+    try:
+        assert L.dba_test_hook(None, 2_000_000, 0) == 0
+        lse, val, idx = dba.project_scan(hd, ed, n_top)
+        assert torch.isnan(lse).all() and (idx == -1).all() and torch.isinf(val).all()
+    finally:
+        assert L.dba_test_hook(None, 0, -1) == 0
+    lse, val, idx = dba.project_scan(hd, ed, n_top)
+    assert torch.isfinite(lse).all() and (idx >= 0).all()
+    B, k = 3, 4
+    st = dba.DbaStepper(B, k, V, 4, constraints=[[[5]], [], [[6, 7]]], dtype=dba.F32, flags=dba.FLAG_FUSED_PROJECTION)
+    st.test_hook(wait_clocks=2_000_000, drop_item=0)
+    st.step_fused(hd[:B * k].contiguous(), ed)
+    with pytest.raises(dba.DbaError) as err:
+        st.finalize()
+    assert err.value.code == 5                   # DBA_ERR_TIMEOUT
+    st.close()
+    st2 = dba.DbaStepper(B, k, V, 4, constraints=[[[5]], [], [[6, 7]]], dtype=dba.F32, flags=dba.FLAG_FUSED_PROJECTION)
+    st2.step_fused(hd[:B * k].contiguous(), ed)
+    st2.finalize()
+    st2.close()
+
+
 def test_argument_errors_are_reported_not_launched(dba):
     mk = lambda **kw: dba.DbaStepper(**{**dict(B=1, k=2, V=50, max_steps=3, constraints=[[[5]]]), **kw})
     for kw, code in [(dict(k=65), 2), (dict(constraints=[[[w] for w in range(4, 69)]], V=100), 2),
