@@ -12,7 +12,7 @@ namespace dba {
 
 namespace {
 
-constexpr int kCandMaxThreads = 1024;      // the host picks 1024, 512 or 256 threads: the most whose scratch fits
+constexpr int kCandMaxThreads = 1024;      // the host picks 1024, 640, 512 or 256 threads: the most whose scratch fits
 
 struct Layout {   // byte offsets into dynamic shared memory
     int cons, parent, lse, mask, active, kind, eos_ok, plen, s2_x, rt_score, rt_w, rt_n, rt_ptr, s1_h, s1_i, stage, merged,
@@ -75,7 +75,7 @@ __device__ __forceinline__ uint64_t merge_top32(uint64_t a, uint64_t b, int lane
     return acc;
 }
 
-// 48 registers: two CTAs of 672 threads (a warp per row at k = 20, and one more) fit an SM.
+// 48 registers: two CTAs of 640 threads (a warp per row at k = 20) fit an SM.
 __global__ void __maxnreg__(48)
 candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const SentCons* __restrict__ cons,
                   Beam cur, Beam nxt, RowTop top, ScanScratch part, const float* __restrict__ lse_in,
@@ -615,8 +615,8 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
 }  // namespace
 
 // Threads per CTA: 1024 when every sentence gets an SM of its own (then only the latency of one CTA counts);
-// otherwise two CTAs share an SM: 640 threads when the beam has more than 15 rows (a warp per row up to k = 19
-// beside the warp that runs the tournament), else 512; fewer if the per-warp scratch would not fit shared memory.
+// otherwise two CTAs share an SM: 640 threads when the beam has more than 15 rows (a warp per row up to k = 20
+// in the phase that works row by row), else 512; fewer if the per-warp scratch would not fit shared memory.
 static int pick_threads(const Dims& d, size_t smem_limit, int sm_count) {
     const int first = d.B <= sm_count ? kCandMaxThreads : (d.k > 15 ? 640 : 512);
     for (int t = first; t > 256; t = t == 640 ? 512 : t >> 1)
