@@ -167,15 +167,16 @@ candidates_kernel(const void* __restrict__ logits, int64_t stride, Dims d, const
     }
     // Up to here only what earlier steps left behind was read (the row scan waited for them before it let
     // this kernel start); from here on the row scan's own results are needed.
-    grid_dependency_wait();
-    __syncthreads();
     const int C = sc.C;
     if (tid < k) s_eos_ok[tid] = __popcll(s_mask[tid]) >= C;   // Section 3.3: end token only once all are met
-    if (!logits)
+    grid_dependency_wait();
+    if (!logits) {
+        __syncthreads();
         for (int q = tid; q < k * kMaxC; q += n_threads) {
             const int h = q >> 6, j = q & 63;
             if (s_kind[h] == 1 && j < C && s2_x[q] != neg_inf()) s2_x[q] = s2_given[(int64_t)(r0 + h) * kMaxC + j];
         }
+    }
     __syncthreads();
 
     // ---- phase A: per row, the k best cells in (score desc, token asc) order ------------------------------
